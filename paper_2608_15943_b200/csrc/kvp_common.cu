@@ -1,0 +1,98 @@
+// Host utilities of the library: status strings, TMA descriptor construction, device status.
+#include <mutex>
+
+#include "kvp_host.h"
+
+namespace kvp {
+
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+}  // namespace
+
+int make_tensor_map(CUtensorMap* out, const void* base, int elem_bytes, int rank, const uint64_t* dims,
+                    const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return KVP_ERR_CUDA;
+  cuuint64_t gdim[5];
+  cuuint64_t gstride[4];
+  cuuint32_t bdim[5];
+  cuuint32_t estride[5];
+  for (int i = 0; i < rank; ++i) {
+    gdim[i] = dims[i];
+    bdim[i] = box[i];
+    estride[i] = 1;
+    if (i + 1 < rank) gstride[i] = strides_bytes[i];
+  }
+  const CUtensorMapDataType dt = elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  const CUresult r = fn(out, dt, cuuint32_t(rank), const_cast<void*>(base), gdim, gstride, bdim, estride,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? KVP_OK : KVP_ERR_CUDA;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+}  // namespace kvp
+
+extern "C" const char* kvp_status_string(int status) {
+  switch (status) {
+    case KVP_OK: return "ok";
+    case KVP_ERR_INVALID_ARG: return "invalid argument";
+    case KVP_ERR_BAD_DONOR: return "bad donor map";
+    case KVP_ERR_UNSUPPORTED: return "unsupported shape, dtype or alignment";
+    case KVP_ERR_WORKSPACE: return "workspace missing or too small";
+    case KVP_ERR_CUDA: return "CUDA error";
+    case KVP_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int kvp_device_status(void) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return KVP_ERR_CUDA;
+  int bad = 0;
+  int v;
+  v = kvp::gemm_read_status();
+  if (v < 0) return KVP_ERR_CUDA;
+  bad |= v;
+  v = kvp::attn_fwd_read_status();
+  if (v < 0) return KVP_ERR_CUDA;
+  bad |= v;
+  v = kvp::attn_bwd_read_status();
+  if (v < 0) return KVP_ERR_CUDA;
+  bad |= v;
+  v = kvp::decode_read_status();
+  if (v < 0) return KVP_ERR_CUDA;
+  bad |= v;
+  return bad ? KVP_ERR_TIMEOUT : KVP_OK;
+}
+
+extern "C" int kvp_gemm(int M, int N, int K, const void* a, int64_t lda, int a_mn, const void* b, int64_t ldb,
+                        int b_mn, void* c, int64_t ldc, int out_f32, kvp_stream_t stream) {
+  kvp::GemmSeg seg{a, b, lda, ldb, K};
+  return kvp::gemm_bf16(M, N, &seg, 1, a_mn ? 1 : 0, b_mn ? 1 : 0, c, ldc, out_f32 ? 1 : 0,
+                        reinterpret_cast<cudaStream_t>(stream));
+}

@@ -1,0 +1,44 @@
+// Host-side helpers shared by the translation units of the library (not part of the C ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/kvp.h"
+
+namespace kvp {
+
+// Builds a tiled TMA descriptor over a row-major bf16/fp32 tensor of up to 4 dimensions.
+// dims[0] is the innermost (contiguous) extent in elements; strides_bytes[i] is the byte stride
+// of dims[i+1].  box[] is the tile copied per request.  swizzle128 selects the 128-byte swizzle
+// (the inner box extent must then span exactly 128 bytes).  Returns KVP_OK or KVP_ERR_CUDA.
+int make_tensor_map(CUtensorMap* out, const void* base, int elem_bytes, int rank, const uint64_t* dims,
+                    const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// One GEMM "segment": C += op(A) * op(B) over this segment's K extent.
+struct GemmSeg {
+  const void* a;   // bf16
+  const void* b;   // bf16
+  int64_t lda;     // elements: row stride of the stored matrix
+  int64_t ldb;
+  int K;
+};
+
+// C[M,N] = sum over segments of A_s * B_s, bf16 inputs, fp32 accumulation in TMEM.
+//   a_mn == 0: A_s stored [M, K] row-major (K-major);  a_mn == 1: stored [K, M] row-major.
+//   b_mn == 0: B_s stored [N, K] row-major (K-major);  b_mn == 1: stored [K, N] row-major.
+//   out_f32: C is fp32 (else bf16); ldc in elements.
+int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32,
+              cudaStream_t stream);
+
+int gemm_read_status();
+int attn_fwd_read_status();
+int attn_bwd_read_status();
+int decode_read_status();
+
+int sm_count();
+
+}  // namespace kvp

@@ -1,0 +1,151 @@
+"""ctypes binding of the C-ABI library (``include/kvp.h``): argument marshalling only.
+
+Every function takes torch tensors (device memory, streams) and passes raw pointers and sizes to
+the entry point of the same name; all computation happens in the library's CUDA kernels.  Importing
+this module loads ``libkvp.so`` and raises if it has not been built -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvp.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_15943_b200.build` (nvcc, sm_100a)")
+lib = C.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_BAD_DONOR, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+PLAN_STOP_ON_NO_IMPROVE, PLAN_STAGE_LOCAL_DONOR = 1, 2
+STOP_TOLERANCE, STOP_BUDGET, STOP_EXHAUSTED, STOP_NO_IMPROVE = range(4)
+PLACE_ARCH_BALANCED, PLACE_UNIFORM, PLACE_BIPOLAR = range(3)
+OP_PROJ_FWD, OP_PROJ_BWD, OP_ATTN_FWD, OP_ATTN_BWD, OP_DECODE = range(5)
+
+EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_plan", "kvp_layer_flops", "kvp_workspace_bytes",
+           "kvp_proj_fwd", "kvp_proj_bwd", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
+           "kvp_gemm", "kvp_decode_workspace_bytes", "kvp_cache_append", "kvp_decode"]
+
+
+class KvpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+lib.kvp_status_string.restype = C.c_char_p
+lib.kvp_status_string.argtypes = [C.c_int]
+
+
+def status_string(status: int) -> str:
+    return lib.kvp_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise KvpError(status, where)
+
+
+def device_status() -> int:
+    """Synchronises and returns the library's device status (OK or ERR_TIMEOUT / ERR_CUDA)."""
+    lib.kvp_device_status.restype = C.c_int
+    return int(lib.kvp_device_status())
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _ptr_array(ts: Sequence[Optional[torch.Tensor]]):
+    arr = (C.c_void_p * len(ts))()
+    for i, t in enumerate(ts):
+        arr[i] = _ptr(t)
+    return arr
+
+
+def _i32_array(xs: Sequence[int]):
+    return (C.c_int32 * len(xs))(*[int(x) for x in xs])
+
+
+def _u64_array(xs: Sequence[int]):
+    return (C.c_uint64 * len(xs))(*[int(x) for x in xs])
+
+
+# ------------------------------------------------------------------------------------------
+# gemm
+# ------------------------------------------------------------------------------------------
+lib.kvp_gemm.restype = C.c_int
+lib.kvp_gemm.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_int64, C.c_int,
+                         C.c_void_p, C.c_int64, C.c_int, C.c_void_p]
+
+
+def gemm(a: torch.Tensor, b: torch.Tensor, c: torch.Tensor, a_mn: bool = False, b_mn: bool = False) -> torch.Tensor:
+    """c[M,N] = A B.  a is stored [M,K] (a_mn False) or [K,M]; b is stored [N,K] (b_mn False) or
+    [K,N]; c is bf16 or fp32, row-major."""
+    M, N = c.shape
+    K = a.shape[0] if a_mn else a.shape[1]
+    _check(lib.kvp_gemm(M, N, K, a.data_ptr(), a.stride(0), int(a_mn), b.data_ptr(), b.stride(0), int(b_mn),
+                        c.data_ptr(), c.stride(0), int(c.dtype == torch.float32), _stream()), "kvp_gemm")
+    return c
+
+
+# ------------------------------------------------------------------------------------------
+# planner (host)
+# ------------------------------------------------------------------------------------------
+class _PlanIn(C.Structure):
+    _fields_ = [("L", C.c_int32), ("P", C.c_int32), ("stage_begin", C.POINTER(C.c_int32)),
+                ("f_full", C.POINTER(C.c_uint64)), ("f_share", C.POINTER(C.c_uint64)),
+                ("stage_extra", C.POINTER(C.c_uint64)), ("eps_num", C.c_uint32), ("eps_den", C.c_uint32),
+                ("max_conv", C.c_int32), ("flags", C.c_uint32), ("alpha_num", C.c_uint32), ("alpha_den", C.c_uint32),
+                ("placement", C.c_int32)]
+
+
+class _PlanOut(C.Structure):
+    _fields_ = [("z", C.POINTER(C.c_uint8)), ("donor", C.POINTER(C.c_int32)), ("stage_flops", C.POINTER(C.c_uint64)),
+                ("stage_ratio", C.POINTER(C.c_double)), ("fir_num", C.c_uint64), ("fir_den", C.c_uint64),
+                ("fir", C.c_double), ("n_conv", C.c_int32), ("stop_reason", C.c_int32)]
+
+
+class _ModelDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("h", "f", "a", "g", "dh", "s", "vocab", "causal_half")]
+
+
+lib.kvp_plan.restype = C.c_int
+lib.kvp_plan.argtypes = [C.POINTER(_PlanIn), C.POINTER(_PlanOut)]
+lib.kvp_layer_flops.restype = C.c_int
+lib.kvp_layer_flops.argtypes = [C.POINTER(_ModelDesc), C.POINTER(C.c_uint64), C.POINTER(C.c_uint64),
+                                C.POINTER(C.c_uint64)]
+
+
+def plan(stage_begin, f_full, f_share, stage_extra, eps=(0, 1), max_conv=0, stop_on_no_improve=False,
+         stage_local_donor=False, alpha=None, placement=PLACE_ARCH_BALANCED) -> dict:
+    """kvp_plan (Algorithm 1).  Returns dict(z, donor, stage, stage_ratio, fir_num, fir_den, fir,
+    n_conv, stop_reason)."""
+    P = len(stage_begin) - 1
+    L = len(f_full)
+    sb, ff, fs, ex = _i32_array(stage_begin), _u64_array(f_full), _u64_array(f_share), _u64_array(stage_extra)
+    z = (C.c_uint8 * L)()
+    donor = (C.c_int32 * L)()
+    st = (C.c_uint64 * P)()
+    ratio = (C.c_double * P)()
+    flags = (PLAN_STOP_ON_NO_IMPROVE if stop_on_no_improve else 0) | (PLAN_STAGE_LOCAL_DONOR if stage_local_donor else 0)
+    an, ad = alpha if alpha else (0, 1)
+    pin = _PlanIn(L, P, sb, ff, fs, ex, eps[0], eps[1], max_conv, flags, an, ad, placement)
+    pout = _PlanOut(z, donor, st, ratio, 0, 0, 0.0, 0, 0)
+    _check(lib.kvp_plan(C.byref(pin), C.byref(pout)), "kvp_plan")
+    return dict(z=list(z), donor=list(donor), stage=list(st), stage_ratio=list(ratio), fir_num=pout.fir_num,
+                fir_den=pout.fir_den, fir=pout.fir, n_conv=pout.n_conv, stop_reason=pout.stop_reason)
+
+
+def layer_flops(h, f, a, g, dh, s, vocab, causal_half=True):
+    """kvp_layer_flops -> (f_full, f_share, f_lm_head), per token, forward."""
+    m = _ModelDesc(h, f, a, g, dh, s, vocab, int(causal_half))
+    o = [C.c_uint64() for _ in range(3)]
+    _check(lib.kvp_layer_flops(C.byref(m), *[C.byref(x) for x in o]), "kvp_layer_flops")
+    return tuple(int(x.value) for x in o)

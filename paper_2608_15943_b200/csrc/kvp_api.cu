@@ -1,1 +1,220 @@
+// C-ABI entry points of the training / prefill path: argument validation and the sequence of
+// kernel launches per layer.  No allocation, no synchronisation.
 #include "kvp_host.h"
+
+namespace kvp {
+int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, const void* k, const void* v, void* o,
+                   float* lse, cudaStream_t stream);
+size_t attn_bwd_workspace(const kvp_shape* s, const int32_t* donor);
+int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
+                 const void* const* k, const void* const* v, const void* const* o, const void* const* d_o,
+                 const float* const* lse, void* const* dq, float* const* dk_sum, float* const* dv_sum, void* ws,
+                 size_t ws_bytes, cudaStream_t stream);
+int cast_f32_to_bf16(const float* src, void* dst, size_t n, cudaStream_t stream);
+
+namespace {
+
+int check_donor(int L, const int32_t* donor) {
+  if (donor == nullptr) return KVP_ERR_INVALID_ARG;
+  for (int l = 0; l < L; ++l) {
+    const int d = donor[l];
+    if (d < 0 || d > l || donor[d] != d) return KVP_ERR_BAD_DONOR;
+  }
+  return KVP_OK;
+}
+
+int check_shape(const kvp_shape* s) {
+  if (s == nullptr) return KVP_ERR_INVALID_ARG;
+  if (s->L < 1 || s->B < 1 || s->S < 1 || s->D < 1 || s->Hq < 1 || s->Hkv < 1) return KVP_ERR_INVALID_ARG;
+  if (s->dtype != KVP_BF16) return KVP_ERR_UNSUPPORTED;
+  if ((s->dh != 64 && s->dh != 128) || s->Hq % s->Hkv != 0 || s->D % 64 != 0) return KVP_ERR_UNSUPPORTED;
+  return KVP_OK;
+}
+
+bool ptrs_ok(const void* const* arr, int L, const int32_t* donor, bool owners_only) {
+  if (arr == nullptr) return false;
+  for (int l = 0; l < L; ++l) {
+    if (owners_only && donor[l] != l) continue;
+    if (arr[l] == nullptr || !aligned16(arr[l])) return false;
+  }
+  return true;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+}  // namespace
+}  // namespace kvp
+
+using namespace kvp;
+
+extern "C" size_t kvp_workspace_bytes(int op, const kvp_shape* s, const int32_t* donor) {
+  if (check_shape(s) != KVP_OK || check_donor(s->L, donor) != KVP_OK) return 0;
+  switch (op) {
+    case KVP_OP_PROJ_BWD:
+      // bf16 copies of one owner's dk_sum and dv_sum
+      return 2 * align256(size_t(s->B) * s->S * s->Hkv * s->dh * 2);
+    case KVP_OP_ATTN_BWD:
+      return attn_bwd_workspace(s, donor);
+    default:
+      return 0;
+  }
+}
+
+extern "C" int kvp_proj_fwd(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
+                            const void* const* wk, const void* const* wv, void* const* q, void* const* k,
+                            void* const* v, void* ws, size_t ws_bytes, kvp_stream_t stream_) {
+  (void)ws;
+  (void)ws_bytes;
+  int rc = check_shape(s);
+  if (rc == KVP_OK) rc = check_donor(s->L, donor);
+  if (rc != KVP_OK) return rc;
+  if (!ptrs_ok(x, s->L, donor, false) || !ptrs_ok(wq, s->L, donor, false) || !ptrs_ok(wk, s->L, donor, true) ||
+      !ptrs_ok(wv, s->L, donor, true) || !ptrs_ok(q, s->L, donor, false) || !ptrs_ok(k, s->L, donor, true) ||
+      !ptrs_ok(v, s->L, donor, true))
+    return KVP_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh, Nkv = s->Hkv * s->dh;
+  for (int l = 0; l < s->L; ++l) {
+    GemmSeg sq{x[l], wq[l], D, D, D};
+    rc = gemm_bf16(T, Nq, &sq, 1, 0, 0, q[l], Nq, 0, stream);
+    if (rc != KVP_OK) return rc;
+    if (donor[l] == l) {  // consumers have no K/V projections (Eq. 3)
+      GemmSeg sk{x[l], wk[l], D, D, D};
+      rc = gemm_bf16(T, Nkv, &sk, 1, 0, 0, k[l], Nkv, 0, stream);
+      if (rc != KVP_OK) return rc;
+      GemmSeg sv{x[l], wv[l], D, D, D};
+      rc = gemm_bf16(T, Nkv, &sv, 1, 0, 0, v[l], Nkv, 0, stream);
+      if (rc != KVP_OK) return rc;
+    }
+  }
+  return KVP_OK;
+}
+
+extern "C" int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
+                            const void* const* wk, const void* const* wv, const void* const* dq,
+                            const float* const* dk_sum, const float* const* dv_sum, float* const* dwq,
+                            float* const* dwk, float* const* dwv, void* const* dx, void* ws, size_t ws_bytes,
+                            kvp_stream_t stream_) {
+  int rc = check_shape(s);
+  if (rc == KVP_OK) rc = check_donor(s->L, donor);
+  if (rc != KVP_OK) return rc;
+  if (!ptrs_ok(x, s->L, donor, false) || !ptrs_ok(wq, s->L, donor, false) || !ptrs_ok(wk, s->L, donor, true) ||
+      !ptrs_ok(wv, s->L, donor, true) || !ptrs_ok(dq, s->L, donor, false) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(dk_sum), s->L, donor, true) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(dv_sum), s->L, donor, true) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(dwq), s->L, donor, false) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(dwk), s->L, donor, true) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(dwv), s->L, donor, true) || !ptrs_ok(dx, s->L, donor, false))
+    return KVP_ERR_INVALID_ARG;
+  const size_t need = kvp_workspace_bytes(KVP_OP_PROJ_BWD, s, donor);
+  if (ws == nullptr || ws_bytes < need || !aligned16(ws)) return KVP_ERR_WORKSPACE;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh, Nkv = s->Hkv * s->dh;
+  const size_t n_kv = size_t(T) * Nkv;
+  uint8_t* dk_bf = reinterpret_cast<uint8_t*>(ws);
+  uint8_t* dv_bf = dk_bf + align256(n_kv * 2);
+  for (int l = 0; l < s->L; ++l) {
+    // dWq = dQ^T X : A = dQ stored [T, Nq] (MN-major for M = Nq), B = X stored [T, D] (MN-major for N = D)
+    GemmSeg swq{dq[l], x[l], Nq, D, T};
+    rc = gemm_bf16(Nq, D, &swq, 1, 1, 1, dwq[l], D, 1, stream);
+    if (rc != KVP_OK) return rc;
+    if (donor[l] == l) {
+      rc = cast_f32_to_bf16(dk_sum[l], dk_bf, n_kv, stream);
+      if (rc == KVP_OK) rc = cast_f32_to_bf16(dv_sum[l], dv_bf, n_kv, stream);
+      if (rc != KVP_OK) return rc;
+      GemmSeg swk{dk_bf, x[l], Nkv, D, T};
+      rc = gemm_bf16(Nkv, D, &swk, 1, 1, 1, dwk[l], D, 1, stream);
+      if (rc != KVP_OK) return rc;
+      GemmSeg swv{dv_bf, x[l], Nkv, D, T};
+      rc = gemm_bf16(Nkv, D, &swv, 1, 1, 1, dwv[l], D, 1, stream);
+      if (rc != KVP_OK) return rc;
+      // dX = dQ Wq + dK Wk + dV Wv in one pass: three K segments into the same accumulator
+      GemmSeg segs[3] = {{dq[l], wq[l], Nq, D, Nq}, {dk_bf, wk[l], Nkv, D, Nkv}, {dv_bf, wv[l], Nkv, D, Nkv}};
+      rc = gemm_bf16(T, D, segs, 3, 0, 1, dx[l], D, 0, stream);
+    } else {
+      GemmSeg sx{dq[l], wq[l], Nq, D, Nq};
+      rc = gemm_bf16(T, D, &sx, 1, 0, 1, dx[l], D, 0, stream);
+    }
+    if (rc != KVP_OK) return rc;
+  }
+  return KVP_OK;
+}
+
+extern "C" int kvp_out_proj_fwd(const kvp_shape* s, const void* const* o, const void* const* wo, void* const* y,
+                                kvp_stream_t stream_) {
+  int rc = check_shape(s);
+  if (rc != KVP_OK) return rc;
+  if (o == nullptr || wo == nullptr || y == nullptr) return KVP_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh;
+  for (int l = 0; l < s->L; ++l) {
+    if (o[l] == nullptr || wo[l] == nullptr || y[l] == nullptr) return KVP_ERR_INVALID_ARG;
+    GemmSeg sg{o[l], wo[l], Nq, Nq, Nq};
+    rc = gemm_bf16(T, D, &sg, 1, 0, 0, y[l], D, 0, stream);
+    if (rc != KVP_OK) return rc;
+  }
+  return KVP_OK;
+}
+
+extern "C" int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const void* const* wo,
+                                const void* const* dy, void* const* d_o, float* const* dwo, kvp_stream_t stream_) {
+  int rc = check_shape(s);
+  if (rc != KVP_OK) return rc;
+  if (o == nullptr || wo == nullptr || dy == nullptr || d_o == nullptr || dwo == nullptr) return KVP_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh;
+  for (int l = 0; l < s->L; ++l) {
+    if (o[l] == nullptr || wo[l] == nullptr || dy[l] == nullptr || d_o[l] == nullptr || dwo[l] == nullptr)
+      return KVP_ERR_INVALID_ARG;
+    // dO = dY Wo : A = dY [T, D] K-major, B = Wo stored [D, Nq] = [K, N] (MN-major)
+    GemmSeg s1{dy[l], wo[l], D, Nq, D};
+    rc = gemm_bf16(T, Nq, &s1, 1, 0, 1, d_o[l], Nq, 0, stream);
+    if (rc != KVP_OK) return rc;
+    // dWo = dY^T O : [D, Nq], both operands stored token-major
+    GemmSeg s2{dy[l], o[l], D, Nq, T};
+    rc = gemm_bf16(D, Nq, &s2, 1, 1, 1, dwo[l], Nq, 1, stream);
+    if (rc != KVP_OK) return rc;
+  }
+  return KVP_OK;
+}
+
+extern "C" int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
+                            const void* const* k, const void* const* v, void* const* o, float* const* lse, void* ws,
+                            size_t ws_bytes, kvp_stream_t stream_) {
+  (void)ws;
+  (void)ws_bytes;
+  int rc = check_shape(s);
+  if (rc == KVP_OK) rc = check_donor(s->L, donor);
+  if (rc != KVP_OK) return rc;
+  if (!ptrs_ok(q, s->L, donor, false) || !ptrs_ok(k, s->L, donor, true) || !ptrs_ok(v, s->L, donor, true) ||
+      !ptrs_ok(o, s->L, donor, false) || !ptrs_ok(reinterpret_cast<const void* const*>(lse), s->L, donor, false))
+    return KVP_ERR_INVALID_ARG;
+  if (scale < 0.f) return KVP_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  for (int l = 0; l < s->L; ++l) {
+    const int d = donor[l];
+    rc = attn_fwd_layer(s, causal, scale, q[l], k[d], v[d], o[l], lse[l], stream);
+    if (rc != KVP_OK) return rc;
+  }
+  return KVP_OK;
+}
+
+extern "C" int kvp_attn_bwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
+                            const void* const* k, const void* const* v, const void* const* o,
+                            const void* const* d_o, const float* const* lse, void* const* dq, float* const* dk_sum,
+                            float* const* dv_sum, void* ws, size_t ws_bytes, kvp_stream_t stream_) {
+  int rc = check_shape(s);
+  if (rc == KVP_OK) rc = check_donor(s->L, donor);
+  if (rc != KVP_OK) return rc;
+  if (!ptrs_ok(q, s->L, donor, false) || !ptrs_ok(k, s->L, donor, true) || !ptrs_ok(v, s->L, donor, true) ||
+      !ptrs_ok(o, s->L, donor, false) || !ptrs_ok(d_o, s->L, donor, false) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(lse), s->L, donor, false) || !ptrs_ok(dq, s->L, donor, false) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(dk_sum), s->L, donor, true) ||
+      !ptrs_ok(reinterpret_cast<const void* const*>(dv_sum), s->L, donor, true))
+    return KVP_ERR_INVALID_ARG;
+  if (scale < 0.f) return KVP_ERR_INVALID_ARG;
+  const size_t need = attn_bwd_workspace(s, donor);
+  if (need > 0 && (ws == nullptr || ws_bytes < need || !aligned16(ws))) return KVP_ERR_WORKSPACE;
+  return attn_bwd_all(s, donor, causal, scale, q, k, v, o, d_o, lse, dq, dk_sum, dv_sum, ws, ws_bytes,
+                      reinterpret_cast<cudaStream_t>(stream_));
+}

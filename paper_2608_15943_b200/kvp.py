@@ -149,3 +149,79 @@ def layer_flops(h, f, a, g, dh, s, vocab, causal_half=True):
     o = [C.c_uint64() for _ in range(3)]
     _check(lib.kvp_layer_flops(C.byref(m), *[C.byref(x) for x in o]), "kvp_layer_flops")
     return tuple(int(x.value) for x in o)
+
+
+# ------------------------------------------------------------------------------------------
+# training / prefill path
+# ------------------------------------------------------------------------------------------
+class Shape(C.Structure):
+    """kvp_shape."""
+    _fields_ = [(n, C.c_int32) for n in ("L", "B", "S", "D", "Hq", "Hkv", "dh", "dtype")]
+
+    def __init__(self, L, B, S, D, Hq, Hkv, dh, dtype=0):
+        super().__init__(L, B, S, D, Hq, Hkv, dh, dtype)
+
+
+_PP = C.POINTER(C.c_void_p)
+lib.kvp_workspace_bytes.restype = C.c_size_t
+lib.kvp_workspace_bytes.argtypes = [C.c_int, C.POINTER(Shape), C.POINTER(C.c_int32)]
+lib.kvp_proj_fwd.restype = C.c_int
+lib.kvp_proj_fwd.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32)] + [_PP] * 7 + [C.c_void_p, C.c_size_t, C.c_void_p]
+lib.kvp_proj_bwd.restype = C.c_int
+lib.kvp_proj_bwd.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32)] + [_PP] * 11 + [C.c_void_p, C.c_size_t, C.c_void_p]
+lib.kvp_out_proj_fwd.restype = C.c_int
+lib.kvp_out_proj_fwd.argtypes = [C.POINTER(Shape)] + [_PP] * 3 + [C.c_void_p]
+lib.kvp_out_proj_bwd.restype = C.c_int
+lib.kvp_out_proj_bwd.argtypes = [C.POINTER(Shape)] + [_PP] * 5 + [C.c_void_p]
+lib.kvp_attn_fwd.restype = C.c_int
+lib.kvp_attn_fwd.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32), C.c_int, C.c_float] + [_PP] * 5 + \
+    [C.c_void_p, C.c_size_t, C.c_void_p]
+lib.kvp_attn_bwd.restype = C.c_int
+lib.kvp_attn_bwd.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32), C.c_int, C.c_float] + [_PP] * 9 + \
+    [C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+def workspace_bytes(op: int, shape: Shape, donor) -> int:
+    return int(lib.kvp_workspace_bytes(op, C.byref(shape), _i32_array(donor)))
+
+
+def _ws(ws: Optional[torch.Tensor]):
+    return (C.c_void_p(_ptr(ws)), 0 if ws is None else ws.numel() * ws.element_size())
+
+
+def proj_fwd(shape, donor, x, wq, wk, wv, q, k, v, ws=None):
+    p, n = _ws(ws)
+    _check(lib.kvp_proj_fwd(C.byref(shape), _i32_array(donor), _ptr_array(x), _ptr_array(wq), _ptr_array(wk),
+                            _ptr_array(wv), _ptr_array(q), _ptr_array(k), _ptr_array(v), p, n, _stream()),
+           "kvp_proj_fwd")
+
+
+def proj_bwd(shape, donor, x, wq, wk, wv, dq, dk_sum, dv_sum, dwq, dwk, dwv, dx, ws):
+    p, n = _ws(ws)
+    _check(lib.kvp_proj_bwd(C.byref(shape), _i32_array(donor), _ptr_array(x), _ptr_array(wq), _ptr_array(wk),
+                            _ptr_array(wv), _ptr_array(dq), _ptr_array(dk_sum), _ptr_array(dv_sum), _ptr_array(dwq),
+                            _ptr_array(dwk), _ptr_array(dwv), _ptr_array(dx), p, n, _stream()), "kvp_proj_bwd")
+
+
+def out_proj_fwd(shape, o, wo, y):
+    _check(lib.kvp_out_proj_fwd(C.byref(shape), _ptr_array(o), _ptr_array(wo), _ptr_array(y), _stream()),
+           "kvp_out_proj_fwd")
+
+
+def out_proj_bwd(shape, o, wo, dy, d_o, dwo):
+    _check(lib.kvp_out_proj_bwd(C.byref(shape), _ptr_array(o), _ptr_array(wo), _ptr_array(dy), _ptr_array(d_o),
+                                _ptr_array(dwo), _stream()), "kvp_out_proj_bwd")
+
+
+def attn_fwd(shape, donor, q, k, v, o, lse, causal=True, scale=0.0, ws=None):
+    p, n = _ws(ws)
+    _check(lib.kvp_attn_fwd(C.byref(shape), _i32_array(donor), int(causal), float(scale), _ptr_array(q),
+                            _ptr_array(k), _ptr_array(v), _ptr_array(o), _ptr_array(lse), p, n, _stream()),
+           "kvp_attn_fwd")
+
+
+def attn_bwd(shape, donor, q, k, v, o, d_o, lse, dq, dk_sum, dv_sum, ws, causal=True, scale=0.0):
+    p, n = _ws(ws)
+    _check(lib.kvp_attn_bwd(C.byref(shape), _i32_array(donor), int(causal), float(scale), _ptr_array(q),
+                            _ptr_array(k), _ptr_array(v), _ptr_array(o), _ptr_array(d_o), _ptr_array(lse),
+                            _ptr_array(dq), _ptr_array(dk_sum), _ptr_array(dv_sum), p, n, _stream()), "kvp_attn_bwd")

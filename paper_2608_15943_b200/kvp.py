@@ -225,3 +225,44 @@ def attn_bwd(shape, donor, q, k, v, o, d_o, lse, dq, dk_sum, dv_sum, ws, causal=
     _check(lib.kvp_attn_bwd(C.byref(shape), _i32_array(donor), int(causal), float(scale), _ptr_array(q),
                             _ptr_array(k), _ptr_array(v), _ptr_array(o), _ptr_array(d_o), _ptr_array(lse),
                             _ptr_array(dq), _ptr_array(dk_sum), _ptr_array(dv_sum), p, n, _stream()), "kvp_attn_bwd")
+
+
+# ------------------------------------------------------------------------------------------
+# decode over the shared paged cache
+# ------------------------------------------------------------------------------------------
+class DecodeDesc(C.Structure):
+    """kvp_decode_desc."""
+    _fields_ = [(n, C.c_int32) for n in ("L", "B", "Hq", "Hkv", "dh", "page_size", "max_pages", "n_pages",
+                                         "num_splits", "dtype")]
+
+    def __init__(self, L, B, Hq, Hkv, dh, page_size, max_pages, n_pages, num_splits=0, dtype=0):
+        super().__init__(L, B, Hq, Hkv, dh, page_size, max_pages, n_pages, num_splits, dtype)
+
+
+lib.kvp_decode_workspace_bytes.restype = C.c_size_t
+lib.kvp_decode_workspace_bytes.argtypes = [C.POINTER(DecodeDesc), C.POINTER(C.c_int32)]
+lib.kvp_cache_append.restype = C.c_int
+lib.kvp_cache_append.argtypes = [C.POINTER(DecodeDesc), C.POINTER(C.c_int32)] + [_PP] * 4 + \
+    [C.c_void_p, C.c_void_p, C.c_void_p]
+lib.kvp_decode.restype = C.c_int
+lib.kvp_decode.argtypes = [C.POINTER(DecodeDesc), C.POINTER(C.c_int32), C.c_float] + [_PP] * 3 + \
+    [C.c_void_p, C.c_void_p] + [_PP] * 2 + [C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+def decode_workspace_bytes(desc: DecodeDesc, donor) -> int:
+    return int(lib.kvp_decode_workspace_bytes(C.byref(desc), _i32_array(donor)))
+
+
+def cache_append(desc, donor, k_new, v_new, k_cache, v_cache, block_table, lengths):
+    _check(lib.kvp_cache_append(C.byref(desc), _i32_array(donor), _ptr_array(k_new), _ptr_array(v_new),
+                                _ptr_array(k_cache), _ptr_array(v_cache), block_table.data_ptr(),
+                                lengths.data_ptr(), _stream()), "kvp_cache_append")
+
+
+def decode(desc, donor, q, k_cache, v_cache, block_table, lengths, o, lse, ws, scale=0.0, layer_begin=0,
+           layer_end=None):
+    p, n = _ws(ws)
+    _check(lib.kvp_decode(C.byref(desc), _i32_array(donor), float(scale), _ptr_array(q), _ptr_array(k_cache),
+                          _ptr_array(v_cache), block_table.data_ptr(), lengths.data_ptr(), _ptr_array(o),
+                          _ptr_array(lse), layer_begin, desc.L if layer_end is None else layer_end, p, n, _stream()),
+           "kvp_decode")

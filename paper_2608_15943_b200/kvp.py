@@ -55,6 +55,9 @@ def device_status() -> int:
 
 
 def _stream() -> C.c_void_p:
+    # Without a device the entry points still validate their arguments (and fail before any launch).
+    if not torch.cuda.is_available():
+        return C.c_void_p(0)
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 

@@ -1,0 +1,430 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle, element by element, on the
+same seeded inputs.  Tolerances for bf16 outputs: rel-L2 <= 1e-2 and max-abs <= 3e-2 (scaled by
+max(1, |ref|_inf) for tensors whose entries exceed 1, i.e. sums over many tokens); LSE within 1e-3.
+Integer / index work (planner, donor map) is bit-exact and tested without a GPU."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as A
+from paper_2608_15943_b200 import synth
+from paper_2608_15943_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+REL, ABS, LSE_TOL = 1e-2, 3e-2, 1e-3
+
+
+@pytest.fixture(scope="module")
+def kvp():
+    from paper_2608_15943_b200 import kvp as mod
+    assert torch.cuda.is_available()
+    return mod
+
+
+def f64(t):
+    return None if t is None else t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def f64l(ts):
+    return [f64(t) for t in ts]
+
+
+def close(name, got, ref, rel=REL, abs_=ABS):
+    got = f64(got) if isinstance(got, torch.Tensor) else np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (name, got.shape, ref.shape)
+    assert np.isfinite(got).all(), f"{name}: non-finite output"
+    diff = np.abs(got - ref)
+    scale = max(1.0, float(np.abs(ref).max()))
+    if np.linalg.norm(ref) > 1e-6 * math.sqrt(ref.size):   # an exactly-zero reference has no relative error
+        rl2 = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        assert rl2 <= rel, f"{name}: rel-L2 {rl2:.3e} > {rel}"
+    assert diff.max() <= abs_ * scale, f"{name}: max-abs {diff.max():.3e} > {abs_ * scale:.3e}"
+
+
+def lse_close(name, got, ref):
+    d = np.abs(f64(got) - ref).max()
+    assert d <= LSE_TOL, f"{name}: LSE differs by {d:.3e}"
+
+
+def run_block(kvp, cfg, t, out, causal=True):
+    """proj fwd -> attn fwd -> attn bwd -> proj bwd through the C ABI."""
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+    dev = t["x"][0].device
+    kvp.proj_fwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["q"], out["k"], out["v"])
+    kvp.attn_fwd(sh, cfg.donor, out["q"], out["k"], out["v"], out["o"], out["lse"], causal=causal)
+    ws = torch.empty(max(kvp.workspace_bytes(kvp.OP_ATTN_BWD, sh, cfg.donor),
+                         kvp.workspace_bytes(kvp.OP_PROJ_BWD, sh, cfg.donor), 256), dtype=torch.uint8, device=dev)
+    kvp.attn_bwd(sh, cfg.donor, out["q"], out["k"], out["v"], out["o"], t["d_o"], out["lse"], out["dq"],
+                 out["dk_sum"], out["dv_sum"], ws, causal=causal)
+    kvp.proj_bwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["dq"], out["dk_sum"], out["dv_sum"],
+                 out["dwq"], out["dwk"], out["dwv"], out["dx"], ws)
+    torch.cuda.synchronize()
+    assert kvp.device_status() == kvp.OK
+    return sh
+
+
+# ---------------------------------------------------------------------------------------------
+# GEMM building block, every operand layout, ragged tiles
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 256, 256), (200, 264, 72), (1, 8, 8), (640, 1032, 520)])
+@pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 0), (1, 1)])
+def test_gemm_all_layouts(kvp, M, N, K, a_mn, b_mn):
+    a = synth.normal((M, K), 7, 1, 1.0, "cuda")
+    b = synth.normal((N, K), 7, 2, 1.0, "cuda")
+    ref = f64(a) @ f64(b).T
+    sa = a.t().contiguous() if a_mn else a
+    sb = b.t().contiguous() if b_mn else b
+    if (sa.stride(0) % 8) or (sb.stride(0) % 8):
+        with pytest.raises(kvp.KvpError):
+            kvp.gemm(sa, sb, torch.empty(M, N, device="cuda"), a_mn, b_mn)
+        return
+    c32 = torch.full((M, N), float("nan"), device="cuda")
+    kvp.gemm(sa, sb, c32, a_mn, b_mn)
+    close("gemm f32", c32, ref, rel=1e-5, abs_=1e-4)
+    c16 = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    kvp.gemm(sa, sb, c16, a_mn, b_mn)
+    close("gemm bf16", c16, A.round_bf16(ref), rel=1e-3, abs_=1e-2)
+    assert kvp.device_status() == kvp.OK
+
+
+# ---------------------------------------------------------------------------------------------
+# C0: the tiny stack, per-op and composed
+# ---------------------------------------------------------------------------------------------
+def test_c0_block_per_op_and_composed(kvp):
+    cfg = W.C0
+    t = W.make_train_inputs(cfg, "cuda")
+    out = W.alloc_train_outputs(cfg, "cuda")
+    run_block(kvp, cfg, t, out)
+    dims = (cfg.B, cfg.S, cfg.Hq, cfg.Hkv, cfg.dh)
+    x, wq, wk, wv, d_o = (f64l(t[n]) for n in ("x", "wq", "wk", "wv", "d_o"))
+    own = cfg.owners()
+
+    # --- per-op: each op against the oracle fed the operands that op consumed ---
+    q, k, v = A.proj_fwd(x, wq, wk, wv, cfg.donor, *dims)
+    for l in range(cfg.L):
+        close(f"q[{l}]", out["q"][l], q[l])
+    for l in own:
+        close(f"k[{l}]", out["k"][l], k[l])
+        close(f"v[{l}]", out["v"][l], v[l])
+        assert out["k"][l] is not None
+    qs, ks, vs = f64l(out["q"]), f64l(out["k"]), f64l(out["v"])
+    o, lse = A.attn_fwd(qs, ks, vs, cfg.donor)
+    for l in range(cfg.L):
+        close(f"o[{l}]", out["o"][l], o[l])
+        lse_close(f"lse[{l}]", out["lse"][l], lse[l])
+    dq, dk, dv = A.attn_bwd(qs, ks, vs, d_o, cfg.donor)
+    for l in range(cfg.L):
+        close(f"dq[{l}]", out["dq"][l], dq[l])
+    for l in own:
+        close(f"dk_sum[{l}]", out["dk_sum"][l], dk[l])
+        close(f"dv_sum[{l}]", out["dv_sum"][l], dv[l])
+    dqs = f64l(out["dq"])
+    dks = [A.round_bf16(f64(a)) if a is not None else None for a in out["dk_sum"]]
+    dvs = [A.round_bf16(f64(a)) if a is not None else None for a in out["dv_sum"]]
+    dwq, dwk, dwv, dx = A.proj_bwd(x, wq, wk, wv, dqs, dks, dvs, cfg.donor)
+    for l in range(cfg.L):
+        close(f"dwq[{l}]", out["dwq"][l], dwq[l])
+        close(f"dx[{l}]", out["dx"][l], dx[l])
+    for l in own:
+        close(f"dwk[{l}]", out["dwk"][l], dwk[l])
+        close(f"dwv[{l}]", out["dwv"][l], dwv[l])
+
+    # --- composed: oracle end to end with bf16 rounding where the interface stores bf16 ---
+    r = A.round_bf16
+    qc = [r(a) for a in q]
+    kc = [r(a) if a is not None else None for a in k]
+    vc = [r(a) if a is not None else None for a in v]
+    oc, lsec = A.attn_fwd(qc, kc, vc, cfg.donor)
+    dqc, dkc, dvc = A.attn_bwd(qc, kc, vc, d_o, cfg.donor)
+    dwqc, dwkc, dwvc, dxc = A.proj_bwd(x, wq, wk, wv, [r(a) for a in dqc],
+                                       [r(a) if a is not None else None for a in dkc],
+                                       [r(a) if a is not None else None for a in dvc], cfg.donor)
+    for l in range(cfg.L):
+        close(f"composed o[{l}]", out["o"][l], oc[l])
+        assert np.abs(f64(out["lse"][l]) - lsec[l]).max() <= 5e-3
+        close(f"composed dq[{l}]", out["dq"][l], dqc[l])
+        close(f"composed dwq[{l}]", out["dwq"][l], dwqc[l])
+        close(f"composed dx[{l}]", out["dx"][l], dxc[l])
+    for l in own:
+        close(f"composed dk_sum[{l}]", out["dk_sum"][l], dkc[l])
+        close(f"composed dv_sum[{l}]", out["dv_sum"][l], dvc[l])
+        close(f"composed dwk[{l}]", out["dwk"][l], dwkc[l])
+        close(f"composed dwv[{l}]", out["dwv"][l], dwvc[l])
+
+
+# ---------------------------------------------------------------------------------------------
+# attention forward / backward over shapes that span several tiles and ragged tails
+# ---------------------------------------------------------------------------------------------
+SHAPES = [
+    # B, S, Hq, Hkv, dh, donor, causal
+    (1, 1, 2, 1, 128, [0], True),
+    (1, 127, 2, 2, 128, [0, 0], True),
+    (2, 129, 4, 2, 64, [0, 0, 2, 2], True),
+    (1, 130, 2, 1, 64, [0, 1], False),
+    (1, 384, 8, 2, 128, [0, 0, 0], True),
+    (2, 300, 4, 4, 128, [0, 1, 1], False),
+    (1, 515, 4, 1, 64, [0, 0], True),
+]
+
+
+def attn_inputs(B, S, Hq, Hkv, dh, donor, seed=11, std=1.0):
+    L = len(donor)
+    q = [synth.normal((B, S, Hq, dh), seed, synth.tid(20, l), std, "cuda") for l in range(L)]
+    k = [synth.normal((B, S, Hkv, dh), seed, synth.tid(21, l), std, "cuda") if donor[l] == l else None for l in range(L)]
+    v = [synth.normal((B, S, Hkv, dh), seed, synth.tid(22, l), 1.0, "cuda") if donor[l] == l else None for l in range(L)]
+    d_o = [synth.normal((B, S, Hq, dh), seed, synth.tid(23, l), 1.0, "cuda") for l in range(L)]
+    return q, k, v, d_o
+
+
+@pytest.mark.parametrize("B,S,Hq,Hkv,dh,donor,causal", SHAPES)
+def test_attention_forward_and_backward_shapes(kvp, B, S, Hq, Hkv, dh, donor, causal):
+    L = len(donor)
+    q, k, v, d_o = attn_inputs(B, S, Hq, Hkv, dh, donor)
+    sh = kvp.Shape(L, B, S, 64, Hq, Hkv, dh)
+    o = [torch.full_like(x, float("nan")) for x in q]
+    lse = [torch.full((B, Hq, S), float("nan"), device="cuda") for _ in range(L)]
+    kvp.attn_fwd(sh, donor, q, k, v, o, lse, causal=causal)
+    ro, rl = A.attn_fwd(f64l(q), f64l(k), f64l(v), donor, causal=causal)
+    for l in range(L):
+        close(f"o[{l}]", o[l], ro[l])
+        lse_close(f"lse[{l}]", lse[l], rl[l])
+    # bit-identical on a second run (the forward has no atomics)
+    o2 = [torch.empty_like(x) for x in q]
+    lse2 = [torch.empty_like(x) for x in lse]
+    kvp.attn_fwd(sh, donor, q, k, v, o2, lse2, causal=causal)
+    for l in range(L):
+        assert torch.equal(o[l], o2[l]) and torch.equal(lse[l], lse2[l])
+
+    dq = [torch.full_like(x, float("nan")) for x in q]
+    dk = [torch.full((B, S, Hkv, dh), float("nan"), device="cuda") if donor[l] == l else None for l in range(L)]
+    dv = [torch.full((B, S, Hkv, dh), float("nan"), device="cuda") if donor[l] == l else None for l in range(L)]
+    ws = torch.empty(kvp.workspace_bytes(kvp.OP_ATTN_BWD, sh, donor), dtype=torch.uint8, device="cuda")
+    kvp.attn_bwd(sh, donor, q, k, v, o, d_o, lse, dq, dk, dv, ws, causal=causal)
+    rdq, rdk, rdv = A.attn_bwd(f64l(q), f64l(k), f64l(v), f64l(d_o), donor, causal=causal)
+    for l in range(L):
+        close(f"dq[{l}]", dq[l], rdq[l])
+        if donor[l] == l:
+            close(f"dk_sum[{l}]", dk[l], rdk[l])
+            close(f"dv_sum[{l}]", dv[l], rdv[l])
+    # too small a workspace is refused, not overrun
+    if ws.numel() > 256:
+        with pytest.raises(kvp.KvpError) as e:
+            kvp.attn_bwd(sh, donor, q, k, v, o, d_o, lse, dq, dk, dv, ws[:256], causal=causal)
+        assert e.value.status == kvp.ERR_WORKSPACE
+    assert kvp.device_status() == kvp.OK
+
+
+def test_attention_peaked_softmax_and_custom_scale(kvp):
+    """Large scores exercise the running-maximum rescale path."""
+    B, S, Hq, Hkv, dh, donor = 1, 640, 2, 1, 128, [0]
+    q, k, v, _ = attn_inputs(B, S, Hq, Hkv, dh, donor, seed=5, std=3.0)
+    sh = kvp.Shape(1, B, S, 64, Hq, Hkv, dh)
+    o = [torch.empty_like(q[0])]
+    lse = [torch.empty(B, Hq, S, device="cuda")]
+    kvp.attn_fwd(sh, donor, q, k, v, o, lse, causal=True, scale=0.2)
+    ro, rl = A.attn_fwd(f64l(q), f64l(k), f64l(v), donor, causal=True, scale=0.2)
+    close("o", o[0], ro[0])
+    lse_close("lse", lse[0], rl[0])
+
+
+# ---------------------------------------------------------------------------------------------
+# decode
+# ---------------------------------------------------------------------------------------------
+def gather_cache(pool, bt_row, n, page):
+    """Dense [n, Hkv, dh] float64 view of one sequence's first n positions."""
+    n_pg = (n + page - 1) // page
+    x = pool[bt_row[:n_pg].long()]                      # [n_pg, Hkv, page, dh]
+    x = x.permute(0, 2, 1, 3).reshape(n_pg * page, pool.shape[1], pool.shape[3])[:n]
+    return f64(x)
+
+
+def decode_reference(q, k_cache, v_cache, bt, lens, donor, page, scale=None):
+    L = len(donor)
+    B = len(lens)
+    cap = max(lens)
+    kd = [None] * L
+    vd = [None] * L
+    for l in range(L):
+        if donor[l] != l:
+            continue
+        Hkv, dh = k_cache[l].shape[1], k_cache[l].shape[3]
+        kd[l] = np.zeros((B, cap, Hkv, dh))
+        vd[l] = np.zeros((B, cap, Hkv, dh))
+        for b in range(B):
+            kd[l][b, :lens[b]] = gather_cache(k_cache[l], bt[b], lens[b], page)
+            vd[l][b, :lens[b]] = gather_cache(v_cache[l], bt[b], lens[b], page)
+    return A.decode_attend(f64l(q), kd, vd, lens, donor, scale)
+
+
+DEC_CASES = [
+    # L, donor, B, Hq, Hkv, dh, page, lens, splits
+    (1, [0], 1, 4, 1, 128, 16, [1], 0),
+    (2, [0, 0], 3, 8, 2, 128, 128, [127, 128, 129], 0),
+    (4, [0, 0, 2, 2], 2, 4, 2, 64, 64, [129, 640], 3),
+    (4, [0, 0, 0, 0], 2, 8, 2, 128, 32, [777, 31], 2),
+    (3, [0, 0, 0], 1, 16, 1, 64, 16, [100], 1),
+    (2, [0, 1], 2, 2, 2, 128, 16, [50, 60], 7),
+    (6, [0, 0, 0, 0, 0, 0], 1, 8, 2, 128, 16, [333], 0),   # six layers on one donor: two passes
+]
+
+
+@pytest.mark.parametrize("L,donor,B,Hq,Hkv,dh,page,lens,ns", DEC_CASES)
+def test_decode_against_oracle(kvp, L, donor, B, Hq, Hkv, dh, page, lens, ns):
+    max_pages = (max(lens) + page - 1) // page + 1
+    n_pages = B * max_pages
+    g = torch.Generator().manual_seed(3)
+    bt = torch.randperm(n_pages, generator=g).int().reshape(B, max_pages).cuda()
+    lengths = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    kc = [synth.normal((n_pages, Hkv, page, dh), 13, synth.tid(7, l), 1.0, "cuda") if donor[l] == l else None
+          for l in range(L)]
+    vc = [synth.normal((n_pages, Hkv, page, dh), 13, synth.tid(8, l), 1.0, "cuda") if donor[l] == l else None
+          for l in range(L)]
+    q = [synth.normal((B, Hq, dh), 13, synth.tid(6, l), 1.0, "cuda") for l in range(L)]
+    desc = kvp.DecodeDesc(L, B, Hq, Hkv, dh, page, max_pages, n_pages, ns)
+    ws = torch.empty(kvp.decode_workspace_bytes(desc, donor), dtype=torch.uint8, device="cuda")
+
+    def run(desc_, bt_, kc_, vc_):
+        o = [torch.full((B, Hq, dh), float("nan"), device="cuda", dtype=torch.bfloat16) for _ in range(L)]
+        lse = [torch.full((B, Hq), float("nan"), device="cuda") for _ in range(L)]
+        w = torch.empty(kvp.decode_workspace_bytes(desc_, donor), dtype=torch.uint8, device="cuda")
+        kvp.decode(desc_, donor, q, kc_, vc_, bt_, lengths, o, lse, w)
+        return o, lse
+
+    o, lse = run(desc, bt, kc, vc)
+    ro, rl = decode_reference(q, kc, vc, bt, lens, donor, page)
+    for l in range(L):
+        close(f"o[{l}]", o[l], ro[l])
+        lse_close(f"lse[{l}]", lse[l], rl[l])
+    # invariant to the number of splits (up to rounding) ...
+    o1, lse1 = run(kvp.DecodeDesc(L, B, Hq, Hkv, dh, page, max_pages, n_pages, 1), bt, kc, vc)
+    for l in range(L):
+        close(f"o[{l}] one split", o1[l], ro[l])
+        assert (lse1[l] - lse[l]).abs().max().item() <= 1e-4
+    # ... and bit-identical under a permutation of the physical pages
+    perm = torch.randperm(n_pages, generator=g).cuda()
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(n_pages, device="cuda")
+    kc2 = [a[inv].contiguous() if a is not None else None for a in kc]   # new page perm[p] holds old page p
+    vc2 = [a[inv].contiguous() if a is not None else None for a in vc]
+    bt2 = perm[bt.long()].int()
+    o2, lse2 = run(desc, bt2, kc2, vc2)
+    for l in range(L):
+        assert torch.equal(o2[l], o[l]) and torch.equal(lse2[l], lse[l])
+    # layer ranges: one layer at a time (sequential use) gives the same values
+    for l in range(L):
+        ol = [torch.zeros_like(x) for x in o]
+        ll = [torch.zeros_like(x) for x in lse]
+        kvp.decode(desc, donor, q, kc, vc, bt, lengths, ol, ll, ws, layer_begin=l, layer_end=l + 1)
+        assert torch.equal(ol[l], o[l]) and torch.equal(ll[l], lse[l])
+    assert kvp.device_status() == kvp.OK
+
+
+def test_c0_prefill_then_16_decode_steps(kvp):
+    """Prefill the tiny stack, move K/V into pages, then 16 decode steps: project the new token,
+    append for owners, attend over the shared cache; compared step by step with the oracle run with
+    bf16 rounding where the interface stores bf16."""
+    cfg = W.C0
+    steps, page = 16, 16
+    t = W.make_train_inputs(cfg, "cuda")
+    out = W.alloc_train_outputs(cfg, "cuda")
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+    kvp.proj_fwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["q"], out["k"], out["v"])
+    own = cfg.owners()
+    max_pages = (cfg.S + steps + page - 1) // page
+    n_pages = cfg.B * max_pages
+    bt = torch.arange(n_pages, dtype=torch.int32, device="cuda").reshape(cfg.B, max_pages)
+    kc = [None] * cfg.L
+    vc = [None] * cfg.L
+    for l in own:
+        for name, pool_list in (("k", kc), ("v", vc)):
+            pool = torch.zeros(n_pages, cfg.Hkv, page, cfg.dh, dtype=torch.bfloat16, device="cuda")
+            src = out[name][l]                                            # [B,S,Hkv,dh]
+            pg = src.reshape(cfg.B, cfg.S // page, page, cfg.Hkv, cfg.dh).permute(0, 1, 3, 2, 4)
+            pool.view(cfg.B, max_pages, cfg.Hkv, page, cfg.dh)[:, :cfg.S // page] = pg
+            pool_list[l] = pool
+    # oracle state: dense caches from the SAME stored bf16 prefill K/V
+    cap = cfg.S + steps
+    okc = [None] * cfg.L
+    ovc = [None] * cfg.L
+    for l in own:
+        okc[l] = np.zeros((cfg.B, cap, cfg.Hkv, cfg.dh))
+        ovc[l] = np.zeros((cfg.B, cap, cfg.Hkv, cfg.dh))
+        okc[l][:, :cfg.S] = f64(out["k"][l])
+        ovc[l][:, :cfg.S] = f64(out["v"][l])
+    olen = [cfg.S] * cfg.B
+    wq, wk, wv = f64l(t["wq"]), f64l(t["wk"]), f64l(t["wv"])
+    desc = kvp.DecodeDesc(cfg.L, cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, page, max_pages, n_pages, 2)
+    ws = torch.empty(kvp.decode_workspace_bytes(desc, cfg.donor), dtype=torch.uint8, device="cuda")
+    dsh = kvp.Shape(cfg.L, cfg.B, 1, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)      # one token per sequence
+    lengths = torch.full((cfg.B,), cfg.S, dtype=torch.int32, device="cuda")
+    for step in range(steps):
+        x_t = [synth.normal((cfg.B, cfg.D), W.SEED, synth.tid(10, l, step), 1.0, "cuda") for l in range(cfg.L)]
+        qn = [torch.empty(cfg.B, 1, cfg.Hq, cfg.dh, dtype=torch.bfloat16, device="cuda") for _ in range(cfg.L)]
+        kn = [torch.empty(cfg.B, 1, cfg.Hkv, cfg.dh, dtype=torch.bfloat16, device="cuda") if l in own else None
+              for l in range(cfg.L)]
+        vn = [torch.empty(cfg.B, 1, cfg.Hkv, cfg.dh, dtype=torch.bfloat16, device="cuda") if l in own else None
+              for l in range(cfg.L)]
+        kvp.proj_fwd(dsh, cfg.donor, x_t, t["wq"], t["wk"], t["wv"], qn, kn, vn)
+        lengths += 1
+        kvp.cache_append(desc, cfg.donor, kn, vn, kc, vc, bt, lengths)
+        o = [torch.empty(cfg.B, cfg.Hq, cfg.dh, dtype=torch.bfloat16, device="cuda") for _ in range(cfg.L)]
+        lse = [torch.empty(cfg.B, cfg.Hq, device="cuda") for _ in range(cfg.L)]
+        kvp.decode(desc, cfg.donor, qn, kc, vc, bt, lengths, o, lse, ws)
+        oq, oo, ol = A.decode_step(f64l(x_t), wq, wk, wv, okc, ovc, olen, cfg.donor, cfg.Hq, cfg.Hkv, cfg.dh,
+                                   store_round=A.round_bf16)
+        for l in range(cfg.L):
+            close(f"step {step} q[{l}]", qn[l].reshape(cfg.B, cfg.Hq, cfg.dh), oq[l], rel=5e-3)
+            close(f"step {step} o[{l}]", o[l], oo[l])
+            assert np.abs(f64(lse[l]) - ol[l]).max() <= 5e-3   # composed: q, k re-rounded on each side
+    # the appended rows landed where the oracle put them
+    for l in own:
+        got = kc[l].view(cfg.B, max_pages, cfg.Hkv, page, cfg.dh).permute(0, 1, 3, 2, 4).reshape(
+            cfg.B, max_pages * page, cfg.Hkv, cfg.dh)[:, cfg.S:cfg.S + steps]
+        close(f"appended k[{l}]", got, okc[l][:, cfg.S:cfg.S + steps], rel=5e-3)
+    assert kvp.device_status() == kvp.OK
+
+
+def test_decode_clamps_out_of_range_lengths(kvp):
+    L, donor, B, Hq, Hkv, dh, page = 1, [0], 2, 4, 1, 128, 16
+    max_pages, n_pages = 4, 8
+    bt = torch.arange(8, dtype=torch.int32, device="cuda").reshape(B, max_pages)
+    kc = [synth.normal((n_pages, Hkv, page, dh), 1, 1, 1.0, "cuda")]
+    vc = [synth.normal((n_pages, Hkv, page, dh), 1, 2, 1.0, "cuda")]
+    q = [synth.normal((B, Hq, dh), 1, 3, 1.0, "cuda")]
+    desc = kvp.DecodeDesc(L, B, Hq, Hkv, dh, page, max_pages, n_pages, 0)
+    ws = torch.empty(kvp.decode_workspace_bytes(desc, donor), dtype=torch.uint8, device="cuda")
+    o = [torch.empty(B, Hq, dh, dtype=torch.bfloat16, device="cuda")]
+    lse = [torch.empty(B, Hq, device="cuda")]
+    lengths = torch.tensor([0, 10 ** 6], dtype=torch.int32, device="cuda")   # both invalid
+    kvp.decode(desc, donor, q, kc, vc, bt, lengths, o, lse, ws)
+    torch.cuda.synchronize()
+    ro, _ = decode_reference(q, kc, vc, bt, [1, max_pages * page], donor, page)
+    close("clamped", o[0], ro[0])
+    assert kvp.device_status() == kvp.OK
+
+
+# ---------------------------------------------------------------------------------------------
+# output projection (stage workload) and its chain rule
+# ---------------------------------------------------------------------------------------------
+def test_output_projection(kvp):
+    cfg = W.TrainCfg("t", 2, 1, 200, 128, 2, 1, 64, [0, 0])
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+    nq = cfg.Hq * cfg.dh
+    o = [synth.normal((cfg.B, cfg.S, cfg.Hq, cfg.dh), 3, synth.tid(30, l), 1.0, "cuda") for l in range(cfg.L)]
+    wo = [synth.normal((cfg.D, nq), 3, synth.tid(31, l), 0.05, "cuda") for l in range(cfg.L)]
+    dy = [synth.normal((cfg.T, cfg.D), 3, synth.tid(32, l), 1.0, "cuda") for l in range(cfg.L)]
+    y = [torch.empty(cfg.T, cfg.D, dtype=torch.bfloat16, device="cuda") for _ in range(cfg.L)]
+    d_o = [torch.empty_like(x) for x in o]
+    dwo = [torch.empty(cfg.D, nq, device="cuda") for _ in range(cfg.L)]
+    kvp.out_proj_fwd(sh, o, wo, y)
+    kvp.out_proj_bwd(sh, o, wo, dy, d_o, dwo)
+    for l in range(cfg.L):
+        close("y", y[l], A.out_proj_fwd(f64(o[l]), f64(wo[l])))
+        rd, rw = A.out_proj_bwd(f64(o[l]), f64(wo[l]), f64(dy[l]))
+        close("d_o", d_o[l], rd)
+        close("dwo", dwo[l], rw)
+    assert kvp.device_status() == kvp.OK

@@ -1,0 +1,551 @@
+#!/usr/bin/env python
+"""Benchmark of the shared-KV attention block on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload train|prefill|decode|stage]
+                    [--impl ours|reference] [--no-decode] [--no-cpu-baseline]
+
+Default (no flags): N=1, the training step of the Llama-like block (8 layers, donor map
+[0,1,2,3,4,4,4,4], batch 2 x 8192 tokens, bf16): Q / K / V projections, causal flash-attention
+forward, backward with the donor-group dK/dV sum, projection backward -- one "step" is one pass
+of all of these over one batch.  The decode workload (32 layers, batch 32, 16k-32k contexts,
+256 steps over the shared paged cache) is timed in the same run and reported under "decode".
+One JSON line is printed by rank 0.  `--impl reference` times the fp64 CPU oracle on a bounded
+sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_15943_b200 import dist as kdist          # noqa: E402
+from paper_2608_15943_b200 import synth                   # noqa: E402
+from paper_2608_15943_b200 import workloads as W          # noqa: E402
+
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = int(vis.split(",")[index]) if vis and vis.split(",")[index].isdigit() else index
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def timed_region(fn, steps, device, sampler_index):
+    """barrier + synchronize, CUDA events around `steps` calls, synchronize + barrier; ms total (max over ranks)."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    kdist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(sampler_index) as cs:
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+    kdist.barrier()
+    ms = kdist.max_over_ranks(e0.elapsed_time(e1), device)
+    return ms, cs.summary()
+
+
+# ---------------------------------------------------------------------------------------------
+# training / prefill / stage workloads
+# ---------------------------------------------------------------------------------------------
+class TrainRunner:
+    def __init__(self, kvp, cfg: W.TrainCfg, device, backward=True, out_proj=False, bucket=True):
+        self.kvp, self.cfg, self.device, self.backward, self.out_proj = kvp, cfg, device, backward, out_proj
+        self.t = W.make_train_inputs(cfg, device, with_out_proj=out_proj)
+        self.out = W.alloc_train_outputs(cfg, device, with_out_proj=out_proj)
+        self.sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+        nq, nkv = cfg.Hq * cfg.dh, cfg.Hkv * cfg.dh
+        own = set(cfg.owners())
+        if backward and bucket:   # weight gradients live in one flat bucket (one all-reduce per step for N > 1)
+            shapes = [(nq, cfg.D)] * cfg.L + [(nkv, cfg.D) if l in own else None for l in range(cfg.L)] * 2
+            if out_proj:
+                shapes += [(cfg.D, nq)] * cfg.L
+            self.bucket = kdist.GradBucket(shapes, device)
+            v = self.bucket.views
+            self.out["dwq"], self.out["dwk"], self.out["dwv"] = v[:cfg.L], v[cfg.L:2 * cfg.L], v[2 * cfg.L:3 * cfg.L]
+            if out_proj:
+                self.out["dwo"] = v[3 * cfg.L:4 * cfg.L]
+        else:
+            self.bucket = None
+        ws = max(kvp.workspace_bytes(kvp.OP_ATTN_BWD, self.sh, cfg.donor),
+                 kvp.workspace_bytes(kvp.OP_PROJ_BWD, self.sh, cfg.donor), 256) if backward else 256
+        self.ws = torch.empty(ws, dtype=torch.uint8, device=device)
+        if out_proj and backward:
+            self.d_o = [torch.empty_like(x) for x in self.out["o"]]
+
+    def step(self, _i=0):
+        k, c, t, o = self.kvp, self.cfg, self.t, self.out
+        k.proj_fwd(self.sh, c.donor, t["x"], t["wq"], t["wk"], t["wv"], o["q"], o["k"], o["v"])
+        k.attn_fwd(self.sh, c.donor, o["q"], o["k"], o["v"], o["o"], o["lse"])
+        if self.out_proj:
+            k.out_proj_fwd(self.sh, o["o"], t["wo"], o["y"])
+        if not self.backward:
+            return
+        d_o = t["d_o"]
+        if self.out_proj:
+            k.out_proj_bwd(self.sh, o["o"], t["wo"], t["dy"], self.d_o, o["dwo"])
+            d_o = self.d_o
+        k.attn_bwd(self.sh, c.donor, o["q"], o["k"], o["v"], o["o"], d_o, o["lse"], o["dq"], o["dk_sum"],
+                   o["dv_sum"], self.ws)
+        k.proj_bwd(self.sh, c.donor, t["x"], t["wq"], t["wk"], t["wv"], o["dq"], o["dk_sum"], o["dv_sum"],
+                   o["dwq"], o["dwk"], o["dwv"], o["dx"], self.ws)
+        if self.bucket is not None:
+            self.bucket.all_reduce()
+
+    def flops(self):
+        c = self.cfg
+        f = c.proj_fwd_flops() + c.attn_fwd_flops()
+        if self.out_proj:
+            f += c.L * 2 * c.T * c.D * c.Hq * c.dh
+        return 3 * f if self.backward else f
+
+    def bwd_kernel_flops_per_step(self):
+        """Algorithmic FLOPs of the attention-backward kernel launches of one step: 4 GEMMs
+        (dV, dP, dQ, dK) of 2*dh per visible (query, key) pair."""
+        c = self.cfg
+        return c.L * 8 * c.dh * (c.S * (c.S + 1) // 2) * c.B * c.Hq
+
+    def fwd_kernel_flops_per_step(self):
+        return self.cfg.attn_fwd_flops()
+
+    # end-to-end: the step's inputs come from pinned host memory, the block's dX goes back
+    def setup_e2e(self):
+        names = ["x", "dy" if self.out_proj else "d_o"] if self.backward else ["x"]
+        self.h_in = {n: [a.cpu().pin_memory() for a in self.t[n]] for n in names}
+        self.h_out = torch.empty_like(self.out["dx"][0] if self.backward else self.out["o"][-1],
+                                      device="cpu").pin_memory()
+        self.h2d = sum(a.numel() * a.element_size() for n in names for a in self.h_in[n])
+        self.d2h = self.h_out.numel() * self.h_out.element_size()
+
+    def step_e2e(self, _i=0):
+        for n, hs in self.h_in.items():
+            for dst, src in zip(self.t[n], hs):
+                dst.copy_(src, non_blocking=True)
+        self.step()
+        self.h_out.copy_(self.out["dx"][0] if self.backward else self.out["o"][-1], non_blocking=True)
+
+
+def cpu_baseline_train(cfg: W.TrainCfg, backward: bool, heads: int = 4, proj_tokens: int = 1024):
+    """The oracle, as it stands, on a bounded exact slice: attention forward (+ backward) of one
+    layer, one sequence, `heads` query heads of one KV group at the full sequence length, and the
+    projections of one owner layer on `proj_tokens` tokens."""
+    from oracle import attention as A
+    S, dh, D = cfg.S, cfg.dh, cfg.D
+    seed = W.SEED
+    q = [synth.normal((1, S, heads, dh), seed, synth.tid(20), 1.0).double().numpy()]
+    k = [synth.normal((1, S, 1, dh), seed, synth.tid(21), 1.0).double().numpy()]
+    v = [synth.normal((1, S, 1, dh), seed, synth.tid(22), 1.0).double().numpy()]
+    g = [synth.normal((1, S, heads, dh), seed, synth.tid(23), 1.0).double().numpy()]
+    nq, nkv = cfg.Hq * dh, cfg.Hkv * dh
+    x = [synth.normal((proj_tokens, D), seed, synth.tid(0), 1.0).double().numpy()]
+    wq = [synth.normal((nq, D), seed, synth.tid(1), 0.02).double().numpy()]
+    wk = [synth.normal((nkv, D), seed, synth.tid(2), 0.02).double().numpy()]
+    wv = [synth.normal((nkv, D), seed, synth.tid(3), 0.02).double().numpy()]
+    t0 = time.perf_counter()
+    A.attn_fwd(q, k, v, [0])
+    qq, kk, vv = A.proj_fwd(x, wq, wk, wv, [0], 1, proj_tokens, cfg.Hq, cfg.Hkv, dh)
+    if backward:
+        A.attn_bwd(q, k, v, g, [0])
+        A.proj_bwd(x, wq, wk, wv, qq, kk, vv, [0])
+    dt = time.perf_counter() - t0
+    flops = 4 * dh * (S * (S + 1) // 2) * heads + 2 * proj_tokens * D * (nq + 2 * nkv)
+    if backward:
+        flops *= 3
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    sample = (f"attention fwd{'+bwd' if backward else ''} of 1 layer x 1 sequence x {heads} query heads (one KV group) "
+              f"at S={S}, plus Q/K/V projections fwd{'+bwd' if backward else ''} of one owner layer on {proj_tokens} tokens; "
+              f"{flops / 1e9:.1f} model GFLOP in {dt:.2f} s")
+    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
+            "seconds": dt}
+
+
+# ---------------------------------------------------------------------------------------------
+# decode workload
+# ---------------------------------------------------------------------------------------------
+class DecodeRunner:
+    def __init__(self, kvp, cfg: W.DecodeCfg, device, n_slots=None, q_sets=4):
+        self.kvp, self.cfg, self.device = kvp, cfg, device
+        self.state = W.make_decode_state(cfg, device, n_slots=n_slots)
+        st = self.state
+        self.desc = kvp.DecodeDesc(cfg.L, cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, cfg.page, cfg.max_pages, st.n_pages, 0)
+        self.ws = torch.empty(kvp.decode_workspace_bytes(self.desc, cfg.donor), dtype=torch.uint8, device=device)
+        self.q = [W.decode_queries(cfg, device, W.SEED, s) for s in range(q_sets)]
+        own = set(cfg.owners())
+        self.k_new = [[synth.normal((cfg.B, cfg.Hkv, cfg.dh), W.SEED, synth.tid(13, l, s), 1.0, device) if l in own
+                       else None for l in range(cfg.L)] for s in range(q_sets)]
+        self.v_new = [[synth.normal((cfg.B, cfg.Hkv, cfg.dh), W.SEED, synth.tid(14, l, s), 1.0, device) if l in own
+                       else None for l in range(cfg.L)] for s in range(q_sets)]
+        self.o = [torch.empty(cfg.B, cfg.Hq, cfg.dh, dtype=torch.bfloat16, device=device) for _ in range(cfg.L)]
+        self.lse = [torch.empty(cfg.B, cfg.Hq, device=device) for _ in range(cfg.L)]
+        self.steps_done = 0
+
+    def reset(self):
+        self.state.lengths.copy_(self.state.lengths0.to(self.device))
+        self.steps_done = 0
+
+    def step(self, i=0):
+        k, c, st = self.kvp, self.cfg, self.state
+        s = i % len(self.q)
+        st.lengths.add_(1)                       # the new token is part of the context it attends to
+        k.cache_append(self.desc, c.donor, self.k_new[s], self.v_new[s], st.k_cache, st.v_cache, st.block_table,
+                       st.lengths)
+        k.decode(self.desc, c.donor, self.q[s], st.k_cache, st.v_cache, st.block_table, st.lengths, self.o,
+                 self.lse, self.ws)
+        self.steps_done += 1
+
+    def setup_e2e(self):
+        c = self.cfg
+        self.h_q = [a.cpu().pin_memory() for a in self.q[0]]
+        self.h_kn = [a.cpu().pin_memory() if a is not None else None for a in self.k_new[0]]
+        self.h_vn = [a.cpu().pin_memory() if a is not None else None for a in self.v_new[0]]
+        self.h_o = [torch.empty_like(a, device="cpu").pin_memory() for a in self.o]
+        nb = lambda xs: sum(a.numel() * a.element_size() for a in xs if a is not None)
+        self.h2d = nb(self.h_q) + nb(self.h_kn) + nb(self.h_vn)
+        self.d2h = nb(self.h_o)
+
+    def step_e2e(self, i=0):
+        for dst, src in zip(self.q[0], self.h_q):
+            dst.copy_(src, non_blocking=True)
+        for dl, sl in ((self.k_new[0], self.h_kn), (self.v_new[0], self.h_vn)):
+            for dst, src in zip(dl, sl):
+                if dst is not None:
+                    dst.copy_(src, non_blocking=True)
+        self.step(0)
+        for dst, src in zip(self.h_o, self.o):
+            dst.copy_(src, non_blocking=True)
+
+
+def cpu_baseline_decode(cfg: W.DecodeCfg, n_seq: int = 16):
+    """The oracle's decode on one stored layer (an owner plus its consumer, if any) and n_seq sequences.
+    Only the time matters here, so the slice is filled by numpy's generator (the seeded table generator
+    is slow on the host)."""
+    from oracle import attention as A
+    lens = [int(x) for x in synth.uniform_ints(cfg.B, cfg.len_lo, cfg.len_hi, W.SEED, synth.tid(9))[:n_seq]]
+    cap = max(lens)
+    members = [l for l in range(cfg.L) if cfg.donor[l] == cfg.owners()[-1]]
+    donor = [0] * len(members)
+    rng = np.random.default_rng(W.SEED)
+    kc = [rng.standard_normal((n_seq, cap, cfg.Hkv, cfg.dh))] + [None] * (len(members) - 1)
+    vc = [rng.standard_normal((n_seq, cap, cfg.Hkv, cfg.dh))] + [None] * (len(members) - 1)
+    q = [rng.standard_normal((n_seq, cfg.Hq, cfg.dh)) for _ in range(len(members))]
+    t0 = time.perf_counter()
+    A.decode_attend(q, kc, vc, lens, donor)
+    dt = time.perf_counter() - t0
+    kv_bytes = sum(lens) * 2 * cfg.Hkv * cfg.dh * 2            # bf16 bytes this slice stands for
+    step_bytes = W.decode_step_bytes(cfg, synth.uniform_ints(cfg.B, cfg.len_lo, cfg.len_hi, W.SEED, synth.tid(9)))
+    est_step_s = dt * step_bytes / kv_bytes
+    return {"value": cfg.B / est_step_s, "unit": "tokens/s", "cores": os.cpu_count() or 1, "kind": "oracle",
+            "sample": f"one stored layer ({len(members)} query layers) x {n_seq} sequences (mean length {sum(lens) // len(lens)}) in {dt:.2f} s, "
+                      f"extrapolated linearly in cache bytes to a full step", "seconds": dt}
+
+
+# ---------------------------------------------------------------------------------------------
+def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
+    if args.workload == "train":
+        cfg, backward, out_proj = W.C2, True, False
+    elif args.workload == "prefill":
+        cfg, backward, out_proj = W.C1, False, False
+    else:
+        raise ValueError(args.workload)
+    runner = TrainRunner(kvp, cfg, device, backward=backward, out_proj=out_proj)
+    for i in range(args.warmup):
+        runner.step(i)
+    torch.cuda.synchronize()
+    status = kvp.device_status()
+    if status != kvp.OK:
+        raise RuntimeError("device status after warm-up: " + kvp.status_string(status))
+    n_groups = len(cfg.owners())
+    main_kernel = kvp.KERNEL_ATTN_BWD if backward else kvp.KERNEL_ATTN_FWD
+    per_step_launches = n_groups if backward else cfg.L
+    l0 = kvp.launch_count()
+    with kvp.KernelTimer(main_kernel, args.steps * per_step_launches) as kt:
+        ms, clocks = timed_region(runner.step, args.steps, device, local_rank)
+    launches = kvp.launch_count() - l0
+    durs = kt.durations_ms()
+    ms_step = ms / args.steps
+    flops = runner.flops()
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    kflops = runner.bwd_kernel_flops_per_step() if backward else runner.fwd_kernel_flops_per_step()
+    k_ms_step = sum(durs) / args.steps
+    achieved = kflops / (k_ms_step * 1e-3) / 1e12
+    peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    roofline = {"bound": "tensor", "kernel": "attn_bwd_kernel<128>" if backward else "attn_fwd_kernel<128>",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": None, "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
+                "launches_per_step": per_step_launches, "kernel_ms_per_step": k_ms_step,
+                "share_of_step": k_ms_step / ms_step,
+                "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS}
+    # end to end through the public API with host buffers
+    runner.setup_e2e()
+    for i in range(2):
+        runner.step_e2e(i)
+    e2e_steps = max(3, min(args.steps, 5))
+    ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
+    e2e_val = world * flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
+    status = kvp.device_status()
+    line = {
+        "metric": "shared-KV attn fwd+bwd TFLOP/s" if backward else "shared-KV attn prefill fwd TFLOP/s",
+        "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": cfg.L, "donor": cfg.donor, "batch_per_gpu": cfg.B,
+                   "global_batch": cfg.B * world, "seq_len": cfg.S, "d_model": cfg.D, "heads": [cfg.Hq, cfg.Hkv],
+                   "head_dim": cfg.dh, "parallelism": f"dp{world}", "l2": "inputs larger than L2 (about 10 GB live)",
+                   "flops": "model count: 3 x forward, causal pairs S(S+1)/2"},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "tokens_per_s": world * cfg.T / (ms_step * 1e-3),
+        "pct_bf16_peak_nominal": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
+        "pct_bf16_peak_measured": 100.0 * value / world / peak,
+        "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": runner.h2d,
+                "d2h_bytes_per_step": runner.d2h, "ms_per_step": ms_e2e / e2e_steps},
+        "roofline": roofline, "device_status": kvp.status_string(status),
+    }
+    del runner
+    torch.cuda.empty_cache()
+    return line, cfg, backward
+
+
+def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, steps=None, warmup=None):
+    cfg = W.C3
+    steps = cfg.steps if steps is None else steps
+    warmup = 3 if warmup is None else warmup
+    free, _total = torch.cuda.mem_get_info()
+    own = len(cfg.owners())
+    lens0 = synth.uniform_ints(cfg.B, cfg.len_lo, cfg.len_hi, W.SEED, synth.tid(9))
+    pages = sum((int(n) + cfg.steps + cfg.page - 1) // cfg.page for n in lens0)
+    per_slot = 2 * pages * cfg.Hkv * cfg.page * cfg.dh * 2
+    n_slots = int(max(1, min(own, (free - (6 << 30)) // per_slot)))
+    runner = DecodeRunner(kvp, cfg, device, n_slots=n_slots)
+    for i in range(warmup):
+        runner.step(i)
+    torch.cuda.synchronize()
+    runner.reset()
+    l0 = kvp.launch_count()
+    with kvp.KernelTimer(kvp.KERNEL_DECODE, steps) as kt:
+        ms, clocks = timed_region(runner.step, steps, device, local_rank)
+    launches = kvp.launch_count() - l0
+    durs = kt.durations_ms()
+    ms_step = ms / steps
+    mean_len = float(lens0.double().mean()) + (steps + 1) / 2.0
+    step_bytes = W.decode_step_bytes(cfg, [mean_len] * cfg.B)
+    k_ms = sum(durs) / len(durs)
+    achieved = step_bytes / (k_ms * 1e-3) / 1e9
+    peak = peaks["hbm_gbs"]
+    unshared_bytes = W.decode_step_bytes(W.C3_UNSHARED, [mean_len] * cfg.B)
+    runner.setup_e2e()
+    runner.reset()
+    for i in range(2):
+        runner.step_e2e(i)
+    e2e_steps = min(steps, 32)
+    ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
+    out = {
+        "metric": "shared-cache decode tokens/s", "value": world * cfg.B / (ms_step * 1e-3), "unit": "tokens/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "hbm_gbs": step_bytes / (ms_step * 1e-3) / 1e9,
+        "config": {"workload": cfg.name, "layers": cfg.L, "stored_layers": own, "batch_per_gpu": cfg.B,
+                   "context": [cfg.len_lo, cfg.len_hi], "page": cfg.page, "heads": [cfg.Hq, cfg.Hkv],
+                   "head_dim": cfg.dh, "physical_layer_pools": n_slots, "mode": "grouped (donor+consumer in one pass)",
+                   "l2": "cache slices far larger than L2", "bytes_per_step": step_bytes,
+                   "bytes_per_step_unshared": unshared_bytes},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": world * cfg.B / (ms_e2e / e2e_steps * 1e-3), "unit": "tokens/s",
+                "h2d_bytes_per_step": runner.h2d, "d2h_bytes_per_step": runner.d2h},
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel<128>", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_kind": f"{peaks_kind} copy bandwidth",
+                     "kernel_ms_per_step": k_ms, "share_of_step": k_ms / ms_step,
+                     "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
+        "device_status": kvp.status_string(kvp.device_status()),
+    }
+    del runner
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_stage(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
+    """Tail pipeline stage of the planned 32-layer decoder: full attention block (Q/K/V projections,
+    attention, output projection) forward + backward, converted (stage-local donor) vs unconverted."""
+    ff, fs, flm = kvp.layer_flops(4096, 11008, 32, 8, 128, 4096, 32000)
+    sb = [4 * i for i in range(9)]
+    plan = kvp.plan(sb, [ff] * 32, [fs] * 32, [0] * 7 + [flm], stop_on_no_improve=True)
+    plan_local = kvp.plan(sb, [ff] * 32, [fs] * 32, [0] * 7 + [flm], stop_on_no_improve=True, stage_local_donor=True)
+    res = {}
+    for cfg in (W.C4_UNCONVERTED, W.C4_STAGE_LOCAL):
+        runner = TrainRunner(kvp, cfg, device, backward=True, out_proj=True)
+        for i in range(args.warmup):
+            runner.step(i)
+        ms, clocks = timed_region(runner.step, args.steps, device, local_rank)
+        res[cfg.name] = {"ms_per_step": ms / args.steps, "tflops": runner.flops() / (ms / args.steps * 1e-3) / 1e12,
+                         "model_flops": runner.flops(), "clocks": clocks}
+        del runner
+        torch.cuda.empty_cache()
+    a, b = res[W.C4_UNCONVERTED.name], res[W.C4_STAGE_LOCAL.name]
+    return {"metric": "tail-stage attention block fwd+bwd ms (converted vs unconverted)", "value": b["ms_per_step"],
+            "unit": "ms", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": b["ms_per_step"],
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "C4-stage", "batch": 8, "seq_len": 4096, "layers": 4,
+                       "plan": {"converted": [l for l, z in enumerate(plan["z"]) if z], "fir": plan["fir"],
+                                "fir_stage_local": plan_local["fir"],
+                                "stage_local_donor": plan_local["donor"][28:]}},
+            "stage": res, "speedup_converted": a["ms_per_step"] / b["ms_per_step"],
+            "flops_ratio_converted": b["model_flops"] / a["model_flops"]}
+
+
+def reference_arm(args, rank, world):
+    """The fp64 CPU oracle on this machine's host cores; each step is a bounded sample of the workload."""
+    if rank != 0:
+        return
+    steps, warmup = args.steps, args.warmup
+    if args.workload == "decode":
+        fn = lambda: cpu_baseline_decode(W.C3, n_seq=1)
+        metric, cfgname = "shared-cache decode tokens/s", W.C3.name
+    else:
+        backward = args.workload != "prefill"
+        cfg = W.C2 if backward else W.C1
+        fn = lambda: cpu_baseline_train(cfg, backward, heads=1, proj_tokens=256)
+        metric = "shared-KV attn fwd+bwd TFLOP/s" if backward else "shared-KV attn prefill fwd TFLOP/s"
+        cfgname = cfg.name
+    for _ in range(min(warmup, 1)):
+        fn()
+    t0 = time.perf_counter()
+    last = None
+    vals = []
+    for _ in range(steps):
+        last = fn()
+        vals.append(last["value"])
+    dt = time.perf_counter() - t0
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": metric, "value": value, "unit": last["unit"], "n_gpus": world,
+            "steps": steps, "warmup": min(warmup, 1), "ms_per_step": dt / steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfgname, "note": "fp64 CPU oracle on a bounded sample per step"},
+            "cpu_baseline": {"value": value, "unit": last["unit"], "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"]},
+            "e2e": {"value": value, "unit": last["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="train", choices=["train", "prefill", "decode", "stage"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-decode", action="store_true", help="skip the decode workload in the default run")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank, local_rank, world = kdist.env_world()
+    if args.impl == "reference":
+        reference_arm(args, rank, world)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the hot path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    kdist.init("nccl")
+    from paper_2608_15943_b200 import kvp     # loads the CUDA library or raises
+    peaks, peaks_kind = measured_peaks()
+
+    if args.workload in ("train", "prefill"):
+        line, cfg, backward = run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
+        if args.workload == "train" and not args.no_decode:
+            try:
+                line["decode"] = run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
+            except Exception as exc:   # report, do not hide: the training line is still valid
+                line["decode"] = {"error": repr(exc)}
+        if rank == 0 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline_train(cfg, backward)
+            if "decode" in line and "error" not in line["decode"]:
+                line["decode"]["cpu_baseline"] = cpu_baseline_decode(W.C3)
+    elif args.workload == "decode":
+        line = run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind,
+                          steps=args.steps if args.steps != 10 else None)
+        if rank == 0 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline_decode(W.C3)
+    else:
+        line = run_stage(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    kdist.barrier()
+
+
+if __name__ == "__main__":
+    main()

@@ -56,6 +56,15 @@ const char* kvp_status_string(int status);
  * gave up on a bounded wait since the last call (the word is cleared), or KVP_ERR_CUDA. */
 int kvp_device_status(void);
 
+/* Benchmark bookkeeping.  kvp_launch_count: kernels launched by this library since it was loaded.
+ * kvp_set_timing_events: record the caller's CUDA events (HOST arrays of n cudaEvent_t, created by
+ * the caller) immediately before and after each of the next n launches of one kernel
+ * (0 GEMM, 1 attention forward, 2 attention backward, 3 decode); n == 0 switches it off.
+ * kvp_timing_events_used: how many pairs have been recorded since.  Not thread-safe. */
+unsigned long long kvp_launch_count(void);
+int kvp_set_timing_events(int kernel, void** starts, void** stops, int n);
+int kvp_timing_events_used(int kernel);
+
 /* ------------------------------------------------------------------------------------------
  * Planner (host only, pure, exact integer arithmetic).
  *

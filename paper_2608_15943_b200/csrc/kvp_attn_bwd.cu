@@ -492,10 +492,13 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     p.scale = sc;
     p.scale_log2 = sc * 1.4426950408889634f;
     dim3 grid((s->S + BT - 1) / BT, s->Hkv, s->B);
+    timing_before(KVP_KERNEL_ATTN_BWD, stream);
     if (dh == 128)
       attn_bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::TOTAL, stream>>>(p);
     else
       attn_bwd_kernel<64><<<grid, BWD_THREADS, BwdSmem<64>::TOTAL, stream>>>(p);
+    timing_after(KVP_KERNEL_ATTN_BWD, stream);
+    note_launch(1 + 2 * n);  // main kernel, n delta pre-passes, n dQ finish passes
     if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
     for (int i = 0; i < n; ++i) {
       const int l = members[i];

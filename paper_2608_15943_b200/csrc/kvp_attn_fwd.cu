@@ -345,6 +345,7 @@ int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, c
   p.scale_log2 = sc * 1.4426950408889634f;
   dim3 grid(s->B * s->Hq, (s->S + BQ - 1) / BQ);
   cudaError_t e;
+  timing_before(KVP_KERNEL_ATTN_FWD, stream);
   if (s->dh == 128) {
     e = cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::TOTAL);
     if (e != cudaSuccess) return KVP_ERR_CUDA;
@@ -356,6 +357,8 @@ int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, c
   } else {
     return KVP_ERR_UNSUPPORTED;
   }
+  timing_after(KVP_KERNEL_ATTN_FWD, stream);
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? KVP_OK : KVP_ERR_CUDA;
 }
 

@@ -1,4 +1,5 @@
 // Host utilities of the library: status strings, TMA descriptor construction, device status.
+#include <atomic>
 #include <mutex>
 
 #include "kvp_host.h"
@@ -46,6 +47,31 @@ int make_tensor_map(CUtensorMap* out, const void* base, int elem_bytes, int rank
   return r == CUDA_SUCCESS ? KVP_OK : KVP_ERR_CUDA;
 }
 
+namespace {
+std::atomic<unsigned long long> g_launches{0};
+struct TimingSlot {
+  cudaEvent_t* starts = nullptr;
+  cudaEvent_t* stops = nullptr;
+  int capacity = 0;
+  int used = 0;
+};
+TimingSlot g_timing[KVP_KERNEL_COUNT];
+}  // namespace
+
+void note_launch(int n) { g_launches.fetch_add(static_cast<unsigned long long>(n), std::memory_order_relaxed); }
+
+void timing_before(int kernel, cudaStream_t stream) {
+  TimingSlot& t = g_timing[kernel];
+  if (t.used < t.capacity) cudaEventRecord(t.starts[t.used], stream);
+}
+void timing_after(int kernel, cudaStream_t stream) {
+  TimingSlot& t = g_timing[kernel];
+  if (t.used < t.capacity) {
+    cudaEventRecord(t.stops[t.used], stream);
+    ++t.used;
+  }
+}
+
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -88,6 +114,24 @@ extern "C" int kvp_device_status(void) {
   if (v < 0) return KVP_ERR_CUDA;
   bad |= v;
   return bad ? KVP_ERR_TIMEOUT : KVP_OK;
+}
+
+extern "C" unsigned long long kvp_launch_count(void) { return kvp::g_launches.load(std::memory_order_relaxed); }
+
+extern "C" int kvp_set_timing_events(int kernel, void** starts, void** stops, int n) {
+  if (kernel < 0 || kernel >= kvp::KVP_KERNEL_COUNT || n < 0 || (n > 0 && (starts == nullptr || stops == nullptr)))
+    return KVP_ERR_INVALID_ARG;
+  kvp::TimingSlot& t = kvp::g_timing[kernel];
+  t.starts = reinterpret_cast<cudaEvent_t*>(starts);
+  t.stops = reinterpret_cast<cudaEvent_t*>(stops);
+  t.capacity = n;
+  t.used = 0;
+  return KVP_OK;
+}
+
+extern "C" int kvp_timing_events_used(int kernel) {
+  if (kernel < 0 || kernel >= kvp::KVP_KERNEL_COUNT) return -1;
+  return kvp::g_timing[kernel].used;
 }
 
 extern "C" int kvp_gemm(int M, int N, int K, const void* a, int64_t lda, int a_mn, const void* b, int64_t ldb,

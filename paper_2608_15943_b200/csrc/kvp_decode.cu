@@ -492,6 +492,7 @@ extern "C" int kvp_cache_append(const kvp_decode_desc* d, const int32_t* donor, 
     }
     if (n == MAX_DEC_GROUPS || (l == d->L && n > 0)) {
       append_kernel<<<dim3(d->B, n), 128, 0, stream>>>(p);
+      note_launch();
       if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
       n = 0;
     }
@@ -564,13 +565,17 @@ extern "C" int kvp_decode(const kvp_decode_desc* d, const int32_t* donor, float 
     }
     dim3 grid(ns, d->B * d->Hkv, n);
     dim3 cgrid(1, d->B * d->Hkv, n);
-    if (d->dh == 128) {
+    timing_before(KVP_KERNEL_DECODE, stream);
+    if (d->dh == 128)
       decode_kernel<128><<<grid, DEC_THREADS, smem, stream>>>(p);
-      decode_combine_kernel<128><<<cgrid, 128, 0, stream>>>(p);
-    } else {
+    else
       decode_kernel<64><<<grid, DEC_THREADS, smem, stream>>>(p);
+    timing_after(KVP_KERNEL_DECODE, stream);
+    if (d->dh == 128)
+      decode_combine_kernel<128><<<cgrid, 128, 0, stream>>>(p);
+    else
       decode_combine_kernel<64><<<cgrid, 128, 0, stream>>>(p);
-    }
+    note_launch(2);
     if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
   }
   return KVP_OK;

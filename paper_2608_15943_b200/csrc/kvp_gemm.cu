@@ -284,15 +284,14 @@ int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, v
     p.map_a[s] = p.map_a[0];
     p.map_b[s] = p.map_b[0];
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GEMM_SMEM)) != cudaSuccess)
-      return KVP_ERR_CUDA;
-    attr_set = true;
-  }
+  if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GEMM_SMEM)) != cudaSuccess)
+    return KVP_ERR_CUDA;
   const int m_tiles = (M + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
   const int grid = min(m_tiles * n_tiles, sm_count());
+  timing_before(KVP_KERNEL_GEMM, stream);
   gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);
+  timing_after(KVP_KERNEL_GEMM, stream);
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? KVP_OK : KVP_ERR_CUDA;
 }
 

@@ -24,6 +24,7 @@ int cast_f32_to_bf16(const float* src, void* dst, size_t n, cudaStream_t stream)
   const int blocks = int(min(size_t(sm_count()) * 8, (n4 + threads - 1) / threads));
   cast_f32_bf16_kernel<<<blocks, threads, 0, stream>>>(reinterpret_cast<const float4*>(src),
                                                        reinterpret_cast<uint2*>(dst), n4);
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? KVP_OK : KVP_ERR_CUDA;
 }
 

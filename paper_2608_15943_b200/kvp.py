@@ -24,7 +24,8 @@ STOP_TOLERANCE, STOP_BUDGET, STOP_EXHAUSTED, STOP_NO_IMPROVE = range(4)
 PLACE_ARCH_BALANCED, PLACE_UNIFORM, PLACE_BIPOLAR = range(3)
 OP_PROJ_FWD, OP_PROJ_BWD, OP_ATTN_FWD, OP_ATTN_BWD, OP_DECODE = range(5)
 
-EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_plan", "kvp_layer_flops", "kvp_workspace_bytes",
+EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events",
+           "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_workspace_bytes",
            "kvp_proj_fwd", "kvp_proj_bwd", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
            "kvp_gemm", "kvp_decode_workspace_bytes", "kvp_cache_append", "kvp_decode"]
 
@@ -269,3 +270,45 @@ def decode(desc, donor, q, k_cache, v_cache, block_table, lengths, o, lse, ws, s
                           _ptr_array(v_cache), block_table.data_ptr(), lengths.data_ptr(), _ptr_array(o),
                           _ptr_array(lse), layer_begin, desc.L if layer_end is None else layer_end, p, n, _stream()),
            "kvp_decode")
+
+
+# ------------------------------------------------------------------------------------------
+# benchmark bookkeeping
+# ------------------------------------------------------------------------------------------
+KERNEL_GEMM, KERNEL_ATTN_FWD, KERNEL_ATTN_BWD, KERNEL_DECODE = range(4)
+lib.kvp_launch_count.restype = C.c_ulonglong
+lib.kvp_set_timing_events.restype = C.c_int
+lib.kvp_set_timing_events.argtypes = [C.c_int, _PP, _PP, C.c_int]
+lib.kvp_timing_events_used.restype = C.c_int
+lib.kvp_timing_events_used.argtypes = [C.c_int]
+
+
+def launch_count() -> int:
+    return int(lib.kvp_launch_count())
+
+
+class KernelTimer:
+    """Records CUDA events around up to n launches of one of the library's kernels and returns the
+    per-launch durations in milliseconds."""
+
+    def __init__(self, kernel: int, n: int):
+        self.kernel, self.n = kernel, n
+        self.starts = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        self.stops = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in self.starts + self.stops:
+            e.record()            # torch creates the underlying event lazily, on first record
+        torch.cuda.synchronize()
+        self._a = (C.c_void_p * n)(*[e.cuda_event for e in self.starts])
+        self._b = (C.c_void_p * n)(*[e.cuda_event for e in self.stops])
+
+    def __enter__(self):
+        _check(lib.kvp_set_timing_events(self.kernel, self._a, self._b, self.n), "kvp_set_timing_events")
+        return self
+
+    def __exit__(self, *exc):
+        self.used = int(lib.kvp_timing_events_used(self.kernel))
+        lib.kvp_set_timing_events(self.kernel, None, None, 0)
+
+    def durations_ms(self):
+        torch.cuda.synchronize()
+        return [self.starts[i].elapsed_time(self.stops[i]) for i in range(self.used)]

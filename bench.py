@@ -317,9 +317,9 @@ def cpu_baseline_decode(cfg: W.DecodeCfg, n_seq: int = 16):
 # ---------------------------------------------------------------------------------------------
 def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
     if args.workload == "train":
-        cfg, backward, out_proj = W.C2, True, False
+        cfg, backward, out_proj = (W.SMALL_TRAIN if args.small else W.C2), True, False
     elif args.workload == "prefill":
-        cfg, backward, out_proj = W.C1, False, False
+        cfg, backward, out_proj = (W.SMALL_TRAIN if args.small else W.C1), False, False
     else:
         raise ValueError(args.workload)
     runner = TrainRunner(kvp, cfg, device, backward=backward, out_proj=out_proj)
@@ -351,12 +351,16 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
                 "share_of_step": k_ms_step / ms_step,
                 "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS}
     # end to end through the public API with host buffers
-    runner.setup_e2e()
-    for i in range(2):
-        runner.step_e2e(i)
-    e2e_steps = max(3, min(args.steps, 5))
-    ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
-    e2e_val = world * flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
+    if args.small:      # profiler capture: the device-timed region is all that is needed
+        ms_e2e, e2e_steps, e2e_val = float("nan"), 1, float("nan")
+        runner.h2d = runner.d2h = 0
+    else:
+        runner.setup_e2e()
+        for i in range(2):
+            runner.step_e2e(i)
+        e2e_steps = max(3, min(args.steps, 5))
+        ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
+        e2e_val = world * flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
     status = kvp.device_status()
     line = {
         "metric": "shared-KV attn fwd+bwd TFLOP/s" if backward else "shared-KV attn prefill fwd TFLOP/s",
@@ -381,7 +385,7 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
 
 
 def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, steps=None, warmup=None):
-    cfg = W.C3
+    cfg = W.SMALL_DECODE if args.small else W.C3
     steps = cfg.steps if steps is None else steps
     warmup = 3 if warmup is None else warmup
     free, _total = torch.cuda.mem_get_info()
@@ -407,12 +411,16 @@ def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, st
     achieved = step_bytes / (k_ms * 1e-3) / 1e9
     peak = peaks["hbm_gbs"]
     unshared_bytes = W.decode_step_bytes(W.C3_UNSHARED, [mean_len] * cfg.B)
-    runner.setup_e2e()
-    runner.reset()
-    for i in range(2):
-        runner.step_e2e(i)
-    e2e_steps = min(steps, 32)
-    ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
+    if args.small:
+        ms_e2e, e2e_steps = float("nan"), 1
+        runner.h2d = runner.d2h = 0
+    else:
+        runner.setup_e2e()
+        runner.reset()
+        for i in range(2):
+            runner.step_e2e(i)
+        e2e_steps = min(steps, 32)
+        ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
     out = {
         "metric": "shared-cache decode tokens/s", "value": world * cfg.B / (ms_step * 1e-3), "unit": "tokens/s",
         "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -509,8 +517,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode workload in the default run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--small", action="store_true",
+                    help="reduced shapes of the same kernels (inputs still larger than L2, under 2 GB on the device) "
+                         "for profiler captures; implies --no-decode for train and --no-cpu-baseline")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" and not args.small else args.warmup
+    if args.small:
+        args.no_decode = args.no_cpu_baseline = True
 
     rank, local_rank, world = kdist.env_world()
     if args.impl == "reference":
@@ -537,7 +550,8 @@ def main():
                 line["decode"]["cpu_baseline"] = cpu_baseline_decode(W.C3)
     elif args.workload == "decode":
         line = run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind,
-                          steps=args.steps if args.steps != 10 else None)
+                          steps=args.steps if (args.steps != 10 or args.small) else None,
+                          warmup=args.warmup if args.small else None)
         if rank == 0 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_decode(W.C3)
     else:

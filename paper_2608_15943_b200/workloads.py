@@ -58,6 +58,8 @@ class TrainCfg:
 C0 = TrainCfg("C0-tiny", 4, 2, 128, 256, 4, 2, 64, [0, 0, 2, 2])
 C1 = TrainCfg("C1-prefill-B4-S4096", 8, 4, 4096, 4096, 32, 8, 128, [0, 1, 2, 3, 4, 4, 4, 4])
 C2 = TrainCfg("C2-train-B2-S8192", 8, 2, 8192, 4096, 32, 8, 128, [0, 1, 2, 3, 4, 4, 4, 4])
+# reduced shapes of the same kernels for profiler captures (inputs larger than L2, < 2 GB live)
+SMALL_TRAIN = TrainCfg("small-train-B1-S4096", 2, 1, 4096, 4096, 32, 8, 128, [0, 0])
 # tail pipeline stage of the 32-layer / PP=8 plan, batch 8 x 4096 tokens
 C4_UNCONVERTED = TrainCfg("C4-stage-unconverted", 4, 8, 4096, 4096, 32, 8, 128, [0, 1, 2, 3])
 C4_STAGE_LOCAL = TrainCfg("C4-stage-local-donor", 4, 8, 4096, 4096, 32, 8, 128, [0, 0, 0, 0])
@@ -134,6 +136,7 @@ def pair_donor(L: int, first_shared: int) -> List[int]:
 
 
 C3 = DecodeCfg("C3-decode-B32-16k-32k", 32, 32, 32, 8, 128, 128, 16384, 32768, pair_donor(32, 16), 256)
+SMALL_DECODE = DecodeCfg("small-decode-B8-8k-16k", 4, 8, 32, 8, 128, 128, 8192, 16384, [0, 0, 2, 2], 8)
 C3_UNSHARED = DecodeCfg("C3-decode-unshared", 32, 32, 32, 8, 128, 128, 16384, 32768, list(range(32)), 256)
 
 

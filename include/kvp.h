@@ -214,6 +214,34 @@ int kvp_decode(const kvp_decode_desc* d, const int32_t* donor, float scale, cons
                const int32_t* lengths, void* const* o, float* const* lse, int layer_begin, int layer_end, void* ws,
                size_t ws_bytes, kvp_stream_t stream);
 
+/* kvp_decode without a workspace argument and without any allocation (the paper has no counterpart:
+ * this is a packaging variant of kvp_decode, same arithmetic, same outputs).
+ *
+ * For callers that cannot obtain device memory where they decode -- a serving loop that has given
+ * the whole device to its cache pool, a plug-in whose host forbids cudaMalloc on its hot path, a
+ * worker that must stay out of the allocator.  The per-split partial results are kept in an array
+ * of KVP_DECODE_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
+ * library holds those bytes until the process exits.
+ *
+ *  - A request whose partials need more than that (kvp_decode_workspace_bytes(d, donor) bytes:
+ *    grows with the number of donor groups, B, Hkv and the split count) is refused with
+ *    KVP_ERR_STATIC_SCRATCH and nothing is launched; lower num_splits, decode a narrower layer
+ *    range per call, or use kvp_decode with your own workspace.
+ *  - No cudaMalloc / cudaFree / allocating library call is made, on any call.
+ *  - The first call on each device looks up the array's device address (with that device current);
+ *    make that first call outside any stream capture.
+ *  - The array is shared by every call and keeps the previous call's contents.  Nothing in it has to
+ *    start at zero: each partial is written by the decode kernel before the combine kernel reads it.
+ *    Two calls whose kernels overlap on the GPU (different streams, or different host threads) race
+ *    on it and corrupt each other's results; serialise them on one stream.
+ *  - All other arguments, layouts and status codes are those of kvp_decode. */
+#define KVP_DECODE_STATIC_SCRATCH_BYTES (16u << 20)
+enum { KVP_ERR_STATIC_SCRATCH = 7 };
+int kvp_decode_static(const kvp_decode_desc* d, const int32_t* donor, float scale, const void* const* q,
+                      const void* const* k_cache, const void* const* v_cache, const int32_t* block_table,
+                      const int32_t* lengths, void* const* o, float* const* lse, int layer_begin, int layer_end,
+                      kvp_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

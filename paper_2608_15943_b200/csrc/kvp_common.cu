@@ -93,6 +93,7 @@ extern "C" const char* kvp_status_string(int status) {
     case KVP_ERR_WORKSPACE: return "workspace missing or too small";
     case KVP_ERR_CUDA: return "CUDA error";
     case KVP_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
+    case KVP_ERR_STATIC_SCRATCH: return "request needs more than the library's built-in scratch array";
     default: return "unknown status";
   }
 }

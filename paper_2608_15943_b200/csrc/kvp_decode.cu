@@ -12,6 +12,8 @@
 // a second small kernel.
 #include <math.h>
 
+#include <mutex>
+
 #include "kvp_host.h"
 #include "kvp_sm100.cuh"
 
@@ -579,4 +581,59 @@ extern "C" int kvp_decode(const kvp_decode_desc* d, const int32_t* donor, float 
     if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
   }
   return KVP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Decode without any caller-provided or allocated scratch.
+//
+// Some callers cannot allocate device memory at the point where they decode: a serving loop that
+// has handed the whole device to its own cache pool and has nothing left to carve a workspace
+// from, a plug-in running inside a host application that forbids cudaMalloc on its hot path, or a
+// worker that must not touch the allocator because another thread holds it.  For them the per-split
+// partial results live in a fixed array that is part of the library image.
+// ---------------------------------------------------------------------------------------------
+namespace kvp {
+namespace {
+
+static __device__ __align__(256) unsigned char g_decode_scratch[KVP_DECODE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {};  // device address of g_decode_scratch, per device ordinal
+
+// The array's name is only a host-side handle here; kernels need its device address, which differs
+// per device and is looked up once with that device current.
+int static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return KVP_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (g_scratch_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_decode_scratch) != cudaSuccess || p == nullptr) return KVP_ERR_CUDA;
+    g_scratch_ptr[dev] = p;
+  }
+  *out = g_scratch_ptr[dev];
+  return KVP_OK;
+}
+
+}  // namespace
+}  // namespace kvp
+
+extern "C" int kvp_decode_static(const kvp_decode_desc* d, const int32_t* donor, float scale, const void* const* q,
+                                 const void* const* k_cache, const void* const* v_cache, const int32_t* block_table,
+                                 const int32_t* lengths, void* const* o, float* const* lse, int layer_begin,
+                                 int layer_end, kvp_stream_t stream) {
+  int rc = check_desc(d);
+  if (rc != KVP_OK) return rc;
+  if (donor == nullptr) return KVP_ERR_INVALID_ARG;
+  for (int l = 0; l < d->L; ++l)
+    if (donor[l] < 0 || donor[l] > l || donor[donor[l]] != donor[l]) return KVP_ERR_BAD_DONOR;
+  const size_t need = kvp_decode_workspace_bytes(d, donor);
+  if (need == 0) return KVP_ERR_UNSUPPORTED;
+  if (need > size_t(KVP_DECODE_STATIC_SCRATCH_BYTES)) return KVP_ERR_STATIC_SCRATCH;
+  void* scratch = nullptr;
+  rc = static_scratch_address(&scratch);
+  if (rc != KVP_OK) return rc;
+  return kvp_decode(d, donor, scale, q, k_cache, v_cache, block_table, lengths, o, lse, layer_begin, layer_end,
+                    scratch, size_t(KVP_DECODE_STATIC_SCRATCH_BYTES), stream);
 }

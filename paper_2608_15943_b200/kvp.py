@@ -27,7 +27,7 @@ OP_PROJ_FWD, OP_PROJ_BWD, OP_ATTN_FWD, OP_ATTN_BWD, OP_DECODE = range(5)
 EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events",
            "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_workspace_bytes",
            "kvp_proj_fwd", "kvp_proj_bwd", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
-           "kvp_gemm", "kvp_decode_workspace_bytes", "kvp_cache_append", "kvp_decode"]
+           "kvp_gemm", "kvp_decode_workspace_bytes", "kvp_cache_append", "kvp_decode", "kvp_decode_static"]
 
 
 class KvpError(RuntimeError):
@@ -312,3 +312,25 @@ class KernelTimer:
     def durations_ms(self):
         torch.cuda.synchronize()
         return [self.starts[i].elapsed_time(self.stops[i]) for i in range(self.used)]
+
+
+# ------------------------------------------------------------------------------------------
+# decode without a workspace: scratch lives in a fixed array inside the library
+# ------------------------------------------------------------------------------------------
+ERR_STATIC_SCRATCH = 7
+DECODE_STATIC_SCRATCH_BYTES = 16 << 20
+lib.kvp_decode_static.restype = C.c_int
+lib.kvp_decode_static.argtypes = [C.POINTER(DecodeDesc), C.POINTER(C.c_int32), C.c_float] + [_PP] * 3 + \
+    [C.c_void_p, C.c_void_p] + [_PP] * 2 + [C.c_int, C.c_int, C.c_void_p]
+
+
+def decode_static(desc, donor, q, k_cache, v_cache, block_table, lengths, o, lse, scale=0.0, layer_begin=0,
+                  layer_end=None):
+    """kvp_decode_static: same results as `decode`, for callers that cannot allocate device memory
+    (no workspace tensor is passed and the library allocates nothing).  Raises KvpError with
+    ERR_STATIC_SCRATCH when the request does not fit the built-in DECODE_STATIC_SCRATCH_BYTES array.
+    Calls share that array, so do not let two of them overlap on the GPU."""
+    _check(lib.kvp_decode_static(C.byref(desc), _i32_array(donor), float(scale), _ptr_array(q), _ptr_array(k_cache),
+                                 _ptr_array(v_cache), block_table.data_ptr(), lengths.data_ptr(), _ptr_array(o),
+                                 _ptr_array(lse), layer_begin, desc.L if layer_end is None else layer_end, _stream()),
+           "kvp_decode_static")

@@ -1,0 +1,234 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times, on sampled
+outputs the oracle can compute one by one (rows of attention are independent given the row's
+query and the visible keys) and on properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as A
+from paper_2608_15943_b200 import synth
+from paper_2608_15943_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+REL, ABS, LSE_TOL = 1e-2, 3e-2, 1e-3
+
+
+def f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def close(name, got, ref, rel=REL, abs_=ABS):
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    assert np.isfinite(got).all(), name
+    scale = max(1.0, float(np.abs(ref).max()))
+    rl2 = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    assert rl2 <= rel, f"{name}: rel-L2 {rl2:.3e}"
+    assert np.abs(got - ref).max() <= abs_ * scale, f"{name}: max-abs {np.abs(got - ref).max():.3e}"
+
+
+def sample_rows(S, rng, n=10):
+    fixed = [0, 1, 127, 128, 129, S // 2 - 1, S // 2, S - 129, S - 128, S - 1]
+    return np.array(sorted(set(fixed + [int(x) for x in rng.integers(0, S, n)])))
+
+
+@pytest.fixture(scope="module")
+def kvp():
+    from paper_2608_15943_b200 import kvp as mod
+    return mod
+
+
+@pytest.fixture(scope="module")
+def c2_run(kvp):
+    """One full training step at C2 (B=2, S=8192, 8 layers, donor [0,1,2,3,4,4,4,4])."""
+    cfg = W.C2
+    t = W.make_train_inputs(cfg, "cuda")
+    out = W.alloc_train_outputs(cfg, "cuda")
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+    ws = torch.empty(max(kvp.workspace_bytes(kvp.OP_ATTN_BWD, sh, cfg.donor),
+                         kvp.workspace_bytes(kvp.OP_PROJ_BWD, sh, cfg.donor)), dtype=torch.uint8, device="cuda")
+    kvp.proj_fwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["q"], out["k"], out["v"])
+    kvp.attn_fwd(sh, cfg.donor, out["q"], out["k"], out["v"], out["o"], out["lse"])
+    kvp.attn_bwd(sh, cfg.donor, out["q"], out["k"], out["v"], out["o"], t["d_o"], out["lse"], out["dq"],
+                 out["dk_sum"], out["dv_sum"], ws)
+    kvp.proj_bwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["dq"], out["dk_sum"], out["dv_sum"],
+                 out["dwq"], out["dwk"], out["dwv"], out["dx"], ws)
+    torch.cuda.synchronize()
+    assert kvp.device_status() == kvp.OK
+    yield cfg, t, out
+    del t, out, ws
+    torch.cuda.empty_cache()
+
+
+def test_c2_projections_sampled_tokens(c2_run):
+    cfg, t, out = c2_run
+    rng = np.random.default_rng(0)
+    toks = sorted(set([0, 127, 128, cfg.T - 1] + [int(x) for x in rng.integers(0, cfg.T, 12)]))
+    for l in (0, 4, 7):
+        x = f64(t["x"][l][toks])
+        close(f"q[{l}]", f64(out["q"][l].reshape(cfg.T, -1)[toks]), x @ f64(t["wq"][l]).T)
+        if cfg.donor[l] == l:
+            close(f"k[{l}]", f64(out["k"][l].reshape(cfg.T, -1)[toks]), x @ f64(t["wk"][l]).T)
+            close(f"v[{l}]", f64(out["v"][l].reshape(cfg.T, -1)[toks]), x @ f64(t["wv"][l]).T)
+        else:
+            assert out["k"][l] is None and out["v"][l] is None
+
+
+def test_c2_attention_forward_sampled_rows(c2_run):
+    cfg, t, out = c2_run
+    rng = np.random.default_rng(1)
+    G = cfg.Hq // cfg.Hkv
+    # every head of KV group 5 of donor 4 and of its consumers, plus scattered heads elsewhere
+    picks = [(l, 1, 5 * G + h) for l in (4, 5, 6, 7) for h in range(G)] + [(0, 0, 0), (2, 1, 31), (3, 0, 17)]
+    for (l, b, hq) in picks:
+        d, hk = cfg.donor[l], hq // G
+        rows = sample_rows(cfg.S, rng)
+        kh, vh = f64(out["k"][d][b, :, hk]), f64(out["v"][d][b, :, hk])
+        ro, rl = A.attn_fwd_rows(f64(out["q"][l][b, rows, hq]), rows, kh, vh)
+        close(f"o[{l},{b},{hq}]", f64(out["o"][l][b, rows, hq]), ro)
+        assert np.abs(f64(out["lse"][l][b, hq, rows]) - rl).max() <= LSE_TOL
+
+
+def _row_backward(q_rows, rows, kh, vh, g_rows, scale):
+    """Oracle arithmetic for single query rows: softmax row, Delta, dS row (chain rule of Eq. 2)."""
+    s = (q_rows @ kh.T) * scale
+    s = np.where(np.arange(kh.shape[0])[None, :] <= rows[:, None], s, -np.inf)
+    m = s.max(axis=1, keepdims=True)
+    p = np.exp(s - m)
+    p /= p.sum(axis=1, keepdims=True)
+    o = p @ vh
+    delta = (g_rows * o).sum(axis=1, keepdims=True)
+    ds = p * (g_rows @ vh.T - delta)
+    return p, ds
+
+
+def test_c2_attention_backward_sampled(c2_run):
+    cfg, t, out = c2_run
+    rng = np.random.default_rng(2)
+    G = cfg.Hq // cfg.Hkv
+    scale = 1.0 / np.sqrt(cfg.dh)
+    # dQ rows, one by one
+    for (l, b, hq) in [(0, 0, 3), (4, 1, 20), (5, 1, 21), (7, 0, 31)]:
+        d, hk = cfg.donor[l], hq // G
+        rows = sample_rows(cfg.S, rng, 6)
+        kh, vh = f64(out["k"][d][b, :, hk]), f64(out["v"][d][b, :, hk])
+        _, ds = _row_backward(f64(out["q"][l][b, rows, hq]), rows, kh, vh, f64(t["d_o"][l][b, rows, hq]), scale)
+        close(f"dq[{l},{b},{hq}]", f64(out["dq"][l][b, rows, hq]), (ds @ kh) * scale)
+    # donor-group dK/dV of layer 4 for the last key rows of one (b, hk): only query rows >= j contribute,
+    # summed over layers 4-7 and the four heads of the group (16 streams)
+    b, hk, j0 = 1, 2, cfg.S - 300
+    rows = np.arange(j0, cfg.S)
+    kh, vh = f64(out["k"][4][b, :, hk]), f64(out["v"][4][b, :, hk])
+    dk = np.zeros((cfg.S - j0, cfg.dh))
+    dv = np.zeros((cfg.S - j0, cfg.dh))
+    for l in (4, 5, 6, 7):
+        for h in range(G):
+            hq = hk * G + h
+            qr, gr = f64(out["q"][l][b, rows, hq]), f64(t["d_o"][l][b, rows, hq])
+            p, ds = _row_backward(qr, rows, kh, vh, gr, scale)
+            dk += (ds[:, j0:].T @ qr) * scale
+            dv += p[:, j0:].T @ gr
+    close("dk_sum[4] tail rows", f64(out["dk_sum"][4][b, j0:, hk]), dk)
+    close("dv_sum[4] tail rows", f64(out["dv_sum"][4][b, j0:, hk]), dv)
+    # property at full size: rows of P sum to one, so sum_j dV[j] = sum over streams and rows of dO
+    for d in (0, 4):
+        members = [l for l in range(cfg.L) if cfg.donor[l] == d]
+        for b in range(cfg.B):
+            got = out["dv_sum"][d][b].double().sum(dim=0)                                   # [Hkv, dh]
+            want = sum(t["d_o"][l][b].double().sum(dim=0).reshape(cfg.Hkv, G, cfg.dh).sum(dim=1) for l in members)
+            rel = ((got - want).norm() / want.norm()).item()
+            assert rel <= 5e-3, f"column-sum property of dV, donor {d}: {rel:.2e}"
+    # owners without consumers received exactly their own gradient: finite and non-trivial
+    for d in cfg.owners():
+        assert torch.isfinite(out["dk_sum"][d]).all() and out["dk_sum"][d].abs().max() > 0
+
+
+def test_c2_projection_backward_sampled(c2_run):
+    cfg, t, out = c2_run
+    rng = np.random.default_rng(3)
+    nq = cfg.Hq * cfg.dh
+    for l in (1, 4, 6):
+        x = f64(t["x"][l])
+        dq = f64(out["dq"][l].reshape(cfg.T, nq))
+        cols = [0, nq - 1] + [int(c) for c in rng.integers(0, nq, 3)]
+        close(f"dwq[{l}]", f64(out["dwq"][l][cols]), dq[:, cols].T @ x)
+        toks = [0, cfg.T - 1] + [int(c) for c in rng.integers(0, cfg.T, 6)]
+        dx = dq[toks] @ f64(t["wq"][l])
+        if cfg.donor[l] == l:
+            dk = A.round_bf16(f64(out["dk_sum"][l].reshape(cfg.T, -1)))
+            dv = A.round_bf16(f64(out["dv_sum"][l].reshape(cfg.T, -1)))
+            kc = [0, dk.shape[1] - 1, 517]
+            close(f"dwk[{l}]", f64(out["dwk"][l][kc]), dk[:, kc].T @ x)
+            close(f"dwv[{l}]", f64(out["dwv"][l][kc]), dv[:, kc].T @ x)
+            dx = dx + dk[toks] @ f64(t["wk"][l]) + dv[toks] @ f64(t["wv"][l])
+        close(f"dx[{l}]", f64(out["dx"][l][toks]), dx)
+
+
+def test_c1_prefill_sampled_rows(kvp):
+    """Prefill configuration (B=4, S=4096): forward only."""
+    cfg = W.C1
+    t = W.make_train_inputs(cfg, "cuda")
+    out = W.alloc_train_outputs(cfg, "cuda")
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+    kvp.proj_fwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["q"], out["k"], out["v"])
+    kvp.attn_fwd(sh, cfg.donor, out["q"], out["k"], out["v"], out["o"], out["lse"])
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(4)
+    G = cfg.Hq // cfg.Hkv
+    for (l, b, hq) in [(0, 0, 0), (4, 3, 12), (5, 3, 13), (6, 2, 14), (7, 1, 15), (3, 2, 31)]:
+        d, hk = cfg.donor[l], hq // G
+        rows = sample_rows(cfg.S, rng)
+        ro, rl = A.attn_fwd_rows(f64(out["q"][l][b, rows, hq]), rows, f64(out["k"][d][b, :, hk]),
+                                 f64(out["v"][d][b, :, hk]))
+        close(f"o[{l},{b},{hq}]", f64(out["o"][l][b, rows, hq]), ro)
+        assert np.abs(f64(out["lse"][l][b, hq, rows]) - rl).max() <= LSE_TOL
+    assert kvp.device_status() == kvp.OK
+    del t, out
+    torch.cuda.empty_cache()
+
+
+def test_c3_decode_full_launch_sampled(kvp):
+    """The long-context decode configuration (32 layers, 24 stored, B=32, 16k-32k contexts) with the
+    stored layers mapped onto two physical pools (same grid, same traffic per launch): sampled
+    (layer, sequence, head) outputs after a few append+decode steps, including donor/consumer pairs."""
+    cfg = W.C3
+    st = W.make_decode_state(cfg, "cuda", n_slots=2)
+    desc = kvp.DecodeDesc(cfg.L, cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, cfg.page, cfg.max_pages, st.n_pages, 0)
+    ws = torch.empty(kvp.decode_workspace_bytes(desc, cfg.donor), dtype=torch.uint8, device="cuda")
+    own = set(cfg.owners())
+    o = [torch.empty(cfg.B, cfg.Hq, cfg.dh, dtype=torch.bfloat16, device="cuda") for _ in range(cfg.L)]
+    lse = [torch.empty(cfg.B, cfg.Hq, device="cuda") for _ in range(cfg.L)]
+    G = cfg.Hq // cfg.Hkv
+    lens = [int(n) for n in st.lengths0]
+    # layers 0 and 2 share physical pool 0 in this test (cyclic mapping): append only to distinct pools
+    for step in range(3):
+        q = W.decode_queries(cfg, "cuda", W.SEED, step)
+        kn = [synth.normal((cfg.B, cfg.Hkv, cfg.dh), W.SEED, synth.tid(13, l, step), 1.0, "cuda") if l in (0, 1)
+              else None for l in range(cfg.L)]
+        vn = [synth.normal((cfg.B, cfg.Hkv, cfg.dh), W.SEED, synth.tid(14, l, step), 1.0, "cuda") if l in (0, 1)
+              else None for l in range(cfg.L)]
+        st.lengths.add_(1)
+        lens = [n + 1 for n in lens]
+        adesc = kvp.DecodeDesc(2, cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, cfg.page, cfg.max_pages, st.n_pages, 0)
+        kvp.cache_append(adesc, [0, 1], kn[:2], vn[:2], st.k_cache[:2], st.v_cache[:2], st.block_table, st.lengths)
+        kvp.decode(desc, cfg.donor, q, st.k_cache, st.v_cache, st.block_table, st.lengths, o, lse, ws)
+    torch.cuda.synchronize()
+    bt = st.block_table.cpu()
+    shortest, longest = int(np.argmin(lens)), int(np.argmax(lens))
+    for (l, b, hq) in [(0, shortest, 0), (1, longest, 9), (15, 3, 31), (16, longest, 4), (17, longest, 5),
+                       (30, shortest, 20), (31, shortest, 23), (31, 7, 16)]:
+        d, hk, n = cfg.donor[l], hq // G, lens[b]
+        n_pg = (n + cfg.page - 1) // cfg.page
+        pages = bt[b, :n_pg].long().cuda()
+        kh = f64(st.k_cache[d][pages, hk].reshape(-1, cfg.dh)[:n])
+        vh = f64(st.v_cache[d][pages, hk].reshape(-1, cfg.dh)[:n])
+        ro, rl = A.attn_fwd_rows(f64(q[l][b, hq:hq + 1]), np.array([n - 1]), kh, vh)
+        close(f"decode o[{l},{b},{hq}]", f64(o[l][b, hq:hq + 1]), ro)
+        assert abs(float(lse[l][b, hq]) - rl[0]) <= LSE_TOL
+    # the appended rows of step 2 are what the last position of layer 0's cache holds
+    b = 5
+    pos = lens[b] - 1
+    page = int(bt[b, pos // cfg.page])
+    assert torch.equal(st.k_cache[0][page, :, pos % cfg.page], kn[0][b])
+    assert torch.equal(st.v_cache[1][page, :, pos % cfg.page], vn[1][b])
+    assert kvp.device_status() == kvp.OK

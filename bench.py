@@ -170,14 +170,11 @@ class TrainRunner:
             f += c.L * 2 * c.T * c.D * c.Hq * c.dh
         return 3 * f if self.backward else f
 
-    def bwd_kernel_flops_per_step(self):
-        """Algorithmic FLOPs of the attention-backward kernel launches of one step: 4 GEMMs
-        (dV, dP, dQ, dK) of 2*dh per visible (query, key) pair."""
+    def gemm_flops(self):
+        """FLOPs of the projection GEMM launches of one step (forward; backward = dW and dX, 2x)."""
         c = self.cfg
-        return c.L * 8 * c.dh * (c.S * (c.S + 1) // 2) * c.B * c.Hq
-
-    def fwd_kernel_flops_per_step(self):
-        return self.cfg.attn_fwd_flops()
+        f = c.proj_fwd_flops() + (c.L * 2 * c.T * c.D * c.Hq * c.dh if self.out_proj else 0)
+        return 3 * f if self.backward else f
 
     # end-to-end: the step's inputs come from pinned host memory, the block's dX goes back
     def setup_e2e(self):
@@ -329,27 +326,44 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
     status = kvp.device_status()
     if status != kvp.OK:
         raise RuntimeError("device status after warm-up: " + kvp.status_string(status))
-    n_groups = len(cfg.owners())
-    main_kernel = kvp.KERNEL_ATTN_BWD if backward else kvp.KERNEL_ATTN_FWD
-    per_step_launches = n_groups if backward else cfg.L
+    n_groups, n_own = len(cfg.owners()), len(cfg.owners())
+    pairs = cfg.S * (cfg.S + 1) // 2
+    unit = 2 * cfg.dh * pairs * cfg.B * cfg.Hq * cfg.L        # one attention GEMM over every layer
+    n_gemm = (cfg.L + 2 * n_own) + ((2 * cfg.L + 2 * n_own) if backward else 0)
+    # kernel -> (launches per step, algorithmic FLOPs per step, executed FLOPs per step)
+    kernels = {"attn_fwd_kernel": (kvp.KERNEL_ATTN_FWD, cfg.L, 2 * unit, 2 * unit),
+               "gemm_kernel": (kvp.KERNEL_GEMM, n_gemm, runner.gemm_flops(), runner.gemm_flops())}
+    if backward:
+        # dK/dV kernel: dV, dP, dK of the model count (it also recomputes S); dQ kernel: dQ (recomputes S, dP)
+        kernels["dkdv_kernel"] = (kvp.KERNEL_ATTN_BWD, n_groups, 3 * unit, 4 * unit)
+        kernels["dq_kernel"] = (kvp.KERNEL_ATTN_BWD_DQ, cfg.L, 1 * unit, 3 * unit)
+    timers = {name: kvp.KernelTimer(kid, args.steps * n) for name, (kid, n, _a, _e) in kernels.items()}
     l0 = kvp.launch_count()
-    with kvp.KernelTimer(main_kernel, args.steps * per_step_launches) as kt:
-        ms, clocks = timed_region(runner.step, args.steps, device, local_rank)
+    for t in timers.values():
+        t.__enter__()
+    ms, clocks = timed_region(runner.step, args.steps, device, local_rank)
+    for t in timers.values():
+        t.__exit__(None, None, None)
     launches = kvp.launch_count() - l0
-    durs = kt.durations_ms()
     ms_step = ms / args.steps
     flops = runner.flops()
     value = world * flops / (ms_step * 1e-3) / 1e12
-    kflops = runner.bwd_kernel_flops_per_step() if backward else runner.fwd_kernel_flops_per_step()
-    k_ms_step = sum(durs) / args.steps
-    achieved = kflops / (k_ms_step * 1e-3) / 1e12
     peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
-    roofline = {"bound": "tensor", "kernel": "attn_bwd_kernel<128>" if backward else "attn_fwd_kernel<128>",
-                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "traffic": None, "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
-                "launches_per_step": per_step_launches, "kernel_ms_per_step": k_ms_step,
-                "share_of_step": k_ms_step / ms_step,
-                "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS}
+    per_kernel = {}
+    for name, (kid, n, algo, execd) in kernels.items():
+        k_ms = sum(timers[name].durations_ms()) / args.steps
+        per_kernel[name] = {"launches_per_step": n, "ms_per_step": k_ms, "share_of_step": k_ms / ms_step,
+                            "algorithmic_tflops": algo / (k_ms * 1e-3) / 1e12,
+                            "executed_tflops": execd / (k_ms * 1e-3) / 1e12}
+    top = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_step"])
+    achieved = per_kernel[top]["algorithmic_tflops"]
+    roofline = {"bound": "tensor", "kernel": top + "<128>", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None, "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
+                "launches_per_step": per_kernel[top]["launches_per_step"],
+                "kernel_ms_per_step": per_kernel[top]["ms_per_step"],
+                "share_of_step": per_kernel[top]["share_of_step"],
+                "executed_tflops": per_kernel[top]["executed_tflops"],
+                "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS, "kernels": per_kernel}
     # end to end through the public API with host buffers
     if args.small:      # profiler capture: the device-timed region is all that is needed
         ms_e2e, e2e_steps, e2e_val = float("nan"), 1, float("nan")

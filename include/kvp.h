@@ -59,7 +59,7 @@ int kvp_device_status(void);
 /* Benchmark bookkeeping.  kvp_launch_count: kernels launched by this library since it was loaded.
  * kvp_set_timing_events: record the caller's CUDA events (HOST arrays of n cudaEvent_t, created by
  * the caller) immediately before and after each of the next n launches of one kernel
- * (0 GEMM, 1 attention forward, 2 attention backward, 3 decode); n == 0 switches it off.
+ * (0 GEMM, 1 attention forward, 2 attention backward dK/dV, 3 decode, 4 attention backward dQ); n == 0 switches it off.
  * kvp_timing_events_used: how many pairs have been recorded since.  Not thread-safe. */
 unsigned long long kvp_launch_count(void);
 int kvp_set_timing_events(int kernel, void** starts, void** stops, int n);
@@ -168,7 +168,8 @@ int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal, float sca
 
 /* Chain rule of Eq. 2-3.  dq[l] (bf16) per layer; dk_sum[d], dv_sum[d] (fp32 [B,S,Hkv,dh], owners
  * only) are the sums over the donor, all its consumers and the Hq/Hkv query heads of each KV head,
- * accumulated in fp32 on chip and written once.  Workspace: kvp_workspace_bytes(KVP_OP_ATTN_BWD). */
+ * accumulated in fp32 on chip and written once.  At most 8 layers may share one donor.
+ * Workspace: kvp_workspace_bytes(KVP_OP_ATTN_BWD). */
 int kvp_attn_bwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
                  const void* const* k, const void* const* v, const void* const* o, const void* const* d_o,
                  const float* const* lse, void* const* dq, float* const* dk_sum, float* const* dv_sum, void* ws,

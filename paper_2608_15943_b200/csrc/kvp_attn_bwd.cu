@@ -1,19 +1,26 @@
-// Flash-attention backward over a donor map (chain rule of Eq. 2-3 of the paper).
+// Flash-attention backward over a donor map (chain rule of Eq. 2-3 of the paper), two kernels:
 //
-// The unit of work is one 128-row K/V tile of one (batch, KV head) of a DONOR layer.  The CTA keeps
-// that K/V tile in shared memory and its dK / dV accumulators in TMEM (fp32) while it walks every
-// query stream that reads the tile: the donor itself and all its consumer layers, the Hq/Hkv query
-// heads of the KV head's group, and every query tile the causal mask lets see the keys.  dK and dV
-// of the donor are therefore summed on chip across layers and heads and written to HBM once.
+//  dkdv_kernel  KV-stationary.  One CTA owns a 128-row K/V tile of one (batch, KV head) of a DONOR
+//               layer, keeps K and V in shared memory and the dK / dV accumulators in TMEM (fp32)
+//               while it walks every query stream that reads the tile: the donor itself and all its
+//               consumer layers, the Hq/Hkv query heads of the KV head's group, and every 64-row query
+//               tile the causal mask lets see the keys.  dK and dV of the donor are therefore summed on
+//               chip across layers and heads and written to HBM once.  Per step, transposed so that TMEM
+//               lane == key row:  S^T = K Q^T, dP^T = V dO^T (tcgen05, operands in shared memory);
+//               P^T = exp2(S^T c - LSE), dS^T = P^T (dP^T - Delta) are written back as bf16 over the
+//               same TMEM columns and fed to dV += P^T dO, dK += dS^T Q as the A operand FROM TMEM --
+//               P and dS never touch shared memory.  Two TMEM buffer sets and two compute warpgroups
+//               alternate, so the tensor pipe works on step n+1 while step n's exponentials run.
 //
-// Per (layer, head, query tile), with everything transposed so that TMEM lane == key row:
-//   S^T  = K Q^T,  dP^T = V dO^T                       (tcgen05, both operands K-major)
-//   P^T  = exp2(S^T c - LSE),  dS^T = P^T (dP^T - Delta)   (one thread per key row)
-//   dV  += P^T dO,   dK += dS^T Q                       (A from shared memory, B MN-major)
-//   dQ   = dS K                                         (A = dS^T read MN-major, B = K MN-major)
-// dQ tiles are added into an fp32 accumulator in the workspace with vector reductions and
-// rounded to bf16 (times the softmax scale) by a small post-pass; Delta = rowsum(dO * O) comes
-// from a pre-pass.
+//  dq_kernel    Q-stationary (like the forward).  One CTA owns a 128-row query tile of one (layer,
+//               batch, query head) and walks the donor's K/V tiles: S = Q K^T, dP = dO V^T,
+//               dS = P (dP - Delta) written as bf16 over dP's TMEM columns, dQ += dS K with dS as the A
+//               operand from TMEM and K as an MN-major B operand.  dQ accumulates in TMEM and is
+//               written once, as bf16, already scaled: no atomics, no fp32 dQ round trip through HBM.
+//
+// Delta = rowsum(dO * O) comes from a small pre-pass.  Recomputing S and dP in both kernels costs
+// two extra GEMMs per tile pair; it removes 64 KB of fp32 reduction traffic per tile pair, which is
+// what bounded the single-kernel form.
 #include <math.h>
 
 #include "kvp_host.h"
@@ -22,37 +29,47 @@
 namespace kvp {
 namespace {
 
-constexpr int BT = 128;            // tile rows for both queries and keys
-constexpr int BWD_THREADS = 192;   // warp 0 TMA, warp 1 MMA, warps 2-5 compute
-constexpr int MAX_GROUP = 8;       // layers of one donor group per launch
-constexpr uint32_t HALF_BYTES = 128 * 128;
+constexpr int BT = 128;    // key rows per tile (both kernels), query rows per tile in dq_kernel
+constexpr int BQ2 = 64;    // query rows per step in dkdv_kernel
+constexpr int MAX_GROUP = 8;  // layers of one donor group per dkdv launch
+constexpr uint32_t HALF_BYTES = 128 * 128;  // [128 rows x 128 B] block
+constexpr uint32_t QHALF_BYTES = 64 * 128;  // [ 64 rows x 128 B] block
 
 __device__ int g_bwd_status;
 
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// =============================================================================================
+// dK / dV
+// =============================================================================================
+constexpr int DKDV_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9 two compute warpgroups
+constexpr int DKDV_STAGES = 4;     // ring of (Q, dO) 64-row tiles
+
 template <int DH>
-struct BwdSmem {
-  static constexpr int TILE = BT * DH * 2;       // K, V, Q, dO tiles
-  static constexpr int PT = BT * BT * 2;         // P^T, dS^T tiles
+struct DkdvSmem {
+  static constexpr int KV_TILE = BT * DH * 2;
+  static constexpr int Q_TILE = BQ2 * DH * 2;
+  static constexpr int STAGE = 2 * Q_TILE;  // Q then dO
   static constexpr int OFF_K = 0;
-  static constexpr int OFF_V = OFF_K + TILE;
-  static constexpr int OFF_Q = OFF_V + TILE;
-  static constexpr int OFF_DO = OFF_Q + TILE;
-  static constexpr int OFF_PT = OFF_DO + TILE;
-  static constexpr int OFF_DST = OFF_PT + PT;
-  static constexpr int OFF_LSE = OFF_DST + PT;   // 128 floats
-  static constexpr int OFF_DELTA = OFF_LSE + 512;
-  static constexpr int OFF_BAR = OFF_DELTA + 512;
-  static constexpr int TOTAL = OFF_BAR + 128 + 1024;
+  static constexpr int OFF_V = OFF_K + KV_TILE;
+  static constexpr int OFF_RING = OFF_V + KV_TILE;
+  static constexpr int OFF_LSE = OFF_RING + DKDV_STAGES * STAGE;  // [2][64] floats
+  static constexpr int OFF_DELTA = OFF_LSE + 2 * BQ2 * 4;
+  static constexpr int OFF_BAR = OFF_DELTA + 2 * BQ2 * 4;
+  static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
 
-struct BwdParams {
-  CUtensorMap map_k, map_v;             // donor K, V: [B,S,Hkv,dh]
-  CUtensorMap map_q[MAX_GROUP];         // per layer of the group: Q  [B,S,Hq,dh]
-  CUtensorMap map_do[MAX_GROUP];        // per layer of the group: dO [B,S,Hq,dh]
-  const float* lse[MAX_GROUP];          // [B,Hq,S]
-  const float* delta[MAX_GROUP];        // [B,Hq,S]
-  float* dq_acc[MAX_GROUP];             // fp32 [B,S,Hq,dh], zero-initialised
-  float* dk_sum;                        // fp32 [B,S,Hkv,dh]
+struct DkdvParams {
+  CUtensorMap map_k, map_v;       // donor K, V: [B,S,Hkv,dh], box rows 128
+  CUtensorMap map_q[MAX_GROUP];   // per layer of the group, box rows 64
+  CUtensorMap map_do[MAX_GROUP];
+  const float* lse[MAX_GROUP];    // [B,Hq,S]
+  const float* delta[MAX_GROUP];  // [B,Hq,S]
+  float* dk_sum;                  // fp32 [B,S,Hkv,dh]
   float* dv_sum;
   int n_layers;
   int B, S, Hq, Hkv;
@@ -61,37 +78,25 @@ struct BwdParams {
   float scale_log2;
 };
 
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
-               : "memory");
-}
-__device__ __forceinline__ void compute_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
 template <int DH>
-__global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_kernel(const __grid_constant__ BwdParams p) {
-  using L = BwdSmem<DH>;
+__global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_constant__ DkdvParams p) {
+  using L = DkdvSmem<DH>;
   constexpr int HALVES = DH / 64;
   constexpr int KSTEPS_DH = DH / 16;
-  constexpr int KSTEPS_T = BT / 16;
+  constexpr int KSTEPS_Q = BQ2 / 16;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* kv_full = bars + 0;
-  uint64_t* qdo_full = bars + 1;   // Q and dO of this iteration landed
-  uint64_t* qdo_empty = bars + 2;  // MMAs that read Q, dO, P^T, dS^T have completed
-  uint64_t* st_full = bars + 3;    // S^T and dP^T are in TMEM
-  uint64_t* pds_ready = bars + 4;  // P^T, dS^T written to shared memory (128 arrivals)
-  uint64_t* dq_full = bars + 5;    // dV, dK, dQ MMAs of this iteration have completed
-  uint64_t* dq_free = bars + 6;    // dQ drained from TMEM (128 arrivals)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-  float* s_lse = reinterpret_cast<float*>(smem + L::OFF_LSE);
-  float* s_delta = reinterpret_cast<float*>(smem + L::OFF_DELTA);
+  uint64_t* q_full = bars + 1;                    // [STAGES]
+  uint64_t* q_empty = q_full + DKDV_STAGES;       // [STAGES]
+  uint64_t* st_full = q_empty + DKDV_STAGES;      // [2]  S^T and dP^T of buffer set b are in TMEM
+  uint64_t* pds_ready = st_full + 2;              // [2]  P^T and dS^T of buffer set b written (128 arrivals)
+  uint64_t* acc_done = pds_ready + 2;             // all MMAs have completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
+  float* s_lse = reinterpret_cast<float*>(smem + L::OFF_LSE);      // [2][64]
+  float* s_delta = reinterpret_cast<float*>(smem + L::OFF_DELTA);  // [2][64]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -102,19 +107,22 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_kernel(const __grid_c
   const int b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
   const int kv0 = jt * BT;
-  const int n_qt = (p.S + BT - 1) / BT;
-  const int qt_first = p.causal ? jt : 0;
+  const int n_qt = (p.S + BQ2 - 1) / BQ2;
+  const int qt_first = p.causal ? (kv0 / BQ2) : 0;
   const int per_stream = n_qt - qt_first;
   const int n_iter = p.n_layers * G * per_stream;
 
   if (threadIdx.x == 0) {
     mbar_init(kv_full, 1);
-    mbar_init(qdo_full, 1);
-    mbar_init(qdo_empty, 1);
-    mbar_init(st_full, 1);
-    mbar_init(pds_ready, 128);
-    mbar_init(dq_full, 1);
-    mbar_init(dq_free, 128);
+    for (int s = 0; s < DKDV_STAGES; ++s) {
+      mbar_init(&q_full[s], 1);
+      mbar_init(&q_empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&st_full[i], 1);
+      mbar_init(&pds_ready[i], 128);
+    }
+    mbar_init(acc_done, 1);
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -125,17 +133,16 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_kernel(const __grid_c
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tm_st = tmem_base;         // S^T, 128 columns
-  const uint32_t tm_dp = tmem_base + 128;   // dP^T, then dQ (aliased)
-  const uint32_t tm_dk = tmem_base + 256;   // DH columns
-  const uint32_t tm_dv = tmem_base + 384;   // DH columns
+  // buffer set i: S^T at [i*128, i*128+64), dP^T at [i*128+64, i*128+128); accumulators above
+  const uint32_t tm_dk = tmem_base + 256;
+  const uint32_t tm_dv = tmem_base + 384;
 
   auto decode_iter = [&](int it, int& li, int& hq, int& q0) {
     const int stream = it / per_stream;
     const int qi = it - stream * per_stream;
     li = stream / G;
     hq = hk * G + (stream - li * G);
-    q0 = (qt_first + qi) * BT;
+    q0 = (qt_first + qi) * BQ2;
   };
 
   if (warp == 0) {
@@ -143,7 +150,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_kernel(const __grid_c
     if (lane == 0) {
       tma_prefetch_desc(&p.map_k);
       tma_prefetch_desc(&p.map_v);
-      mbar_expect_tx(kv_full, 2 * L::TILE);
+      mbar_expect_tx(kv_full, 2 * L::KV_TILE);
 #pragma unroll
       for (int h = 0; h < HALVES; ++h) {
         tma_load_4d(smem + L::OFF_K + h * HALF_BYTES, &p.map_k, kv_full, h * 64, hk, kv0, b);
@@ -152,180 +159,414 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) attn_bwd_kernel(const __grid_c
       for (int it = 0; it < n_iter; ++it) {
         int li, hq, q0;
         decode_iter(it, li, hq, q0);
-        if (!mbar_wait(qdo_empty, (it & 1) ^ 1, err)) break;
-        mbar_expect_tx(qdo_full, 2 * L::TILE);
+        const int s = it % DKDV_STAGES;
+        const uint32_t ph = (it / DKDV_STAGES) & 1;
+        if (!mbar_wait(&q_empty[s], ph ^ 1, err)) break;
+        mbar_expect_tx(&q_full[s], L::STAGE);
+        uint8_t* dst = smem + L::OFF_RING + s * L::STAGE;
 #pragma unroll
         for (int h = 0; h < HALVES; ++h) {
-          tma_load_4d(smem + L::OFF_Q + h * HALF_BYTES, &p.map_q[li], qdo_full, h * 64, hq, q0, b);
-          tma_load_4d(smem + L::OFF_DO + h * HALF_BYTES, &p.map_do[li], qdo_full, h * 64, hq, q0, b);
+          tma_load_4d(dst + h * QHALF_BYTES, &p.map_q[li], &q_full[s], h * 64, hq, q0, b);
+          tma_load_4d(dst + L::Q_TILE + h * QHALF_BYTES, &p.map_do[li], &q_full[s], h * 64, hq, q0, b);
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc_st = umma_idesc_bf16(BT, BT, 0, 0);
-      constexpr uint32_t idesc_acc = umma_idesc_bf16(BT, DH, 0, 1);
-      constexpr uint32_t idesc_dq = umma_idesc_bf16(BT, DH, 1, 1);
+      constexpr uint32_t idesc_st = umma_idesc_bf16(BT, BQ2, 0, 0);   // [128 keys x 64 queries]
+      constexpr uint32_t idesc_acc = umma_idesc_bf16(BT, DH, 0, 1);   // A from TMEM, B MN-major
       const uint32_t sk = smem_u32(smem + L::OFF_K), sv = smem_u32(smem + L::OFF_V);
-      const uint32_t sq = smem_u32(smem + L::OFF_Q), sdo = smem_u32(smem + L::OFF_DO);
-      const uint32_t spt = smem_u32(smem + L::OFF_PT), sdst = smem_u32(smem + L::OFF_DST);
       bool ok = mbar_wait(kv_full, 0, err);
+      auto issue_scores = [&](int it) -> bool {
+        const int s = it % DKDV_STAGES;
+        if (!mbar_wait(&q_full[s], (it / DKDV_STAGES) & 1, err)) return false;
+        tc_fence_after_sync();
+        const uint32_t sq = smem_u32(smem + L::OFF_RING + s * L::STAGE);
+        const uint32_t sdo = sq + L::Q_TILE;
+        const uint32_t tm = tmem_base + (it & 1) * 128;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
+          const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
+          const uint32_t offb = (ks / 4) * QHALF_BYTES + (ks % 4) * 32;
+          umma_ss(tm, smem_desc_sw128(sk + offa, 0, 1024), smem_desc_sw128(sq + offb, 0, 1024), idesc_st, ks != 0);
+        }
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
+          const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
+          const uint32_t offb = (ks / 4) * QHALF_BYTES + (ks % 4) * 32;
+          umma_ss(tm + 64, smem_desc_sw128(sv + offa, 0, 1024), smem_desc_sw128(sdo + offb, 0, 1024), idesc_st,
+                  ks != 0);
+        }
+        umma_commit(&st_full[it & 1]);
+        return true;
+      };
+      if (ok && n_iter > 0) ok = issue_scores(0);
       for (int it = 0; it < n_iter && ok; ++it) {
-        const uint32_t ph = it & 1;
-        if (!mbar_wait(qdo_full, ph, err)) break;
-        // S^T may be overwritten once the compute warps have read the previous one (pds_ready of
-        // it-1, waited below); dP^T / dQ columns once dQ of it-1 has been drained.
-        if (it > 0 && !mbar_wait(dq_free, ph ^ 1, err)) break;
+        // scores of the next step go to the other buffer set; its previous readers (the accumulate
+        // MMAs of step it-1) precede this in the in-order tensor pipe
+        if (it + 1 < n_iter && !issue_scores(it + 1)) { ok = false; break; }
+        if (!mbar_wait(&pds_ready[it & 1], (it >> 1) & 1, err)) { ok = false; break; }
         tc_fence_after_sync();
+        const int s = it % DKDV_STAGES;
+        const uint32_t sq = smem_u32(smem + L::OFF_RING + s * L::STAGE);
+        const uint32_t sdo = sq + L::Q_TILE;
+        const uint32_t tm = tmem_base + (it & 1) * 128;
 #pragma unroll
-        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
-          const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss(tm_st, smem_desc_sw128(sk + off, 0, 1024), smem_desc_sw128(sq + off, 0, 1024), idesc_st, ks != 0);
-        }
+        for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dV += P^T dO
+          umma_ts(tm_dv, tm + ks * 8, smem_desc_sw128(sdo + ks * 2048, QHALF_BYTES, 1024), idesc_acc, (it | ks) != 0);
 #pragma unroll
-        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
-          const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss(tm_dp, smem_desc_sw128(sv + off, 0, 1024), smem_desc_sw128(sdo + off, 0, 1024), idesc_st, ks != 0);
-        }
-        umma_commit(st_full);
-        if (!mbar_wait(pds_ready, ph, err)) break;
-        tc_fence_after_sync();
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS_T; ++ks) {  // dV += P^T dO
-          const uint64_t da = smem_desc_sw128(spt + (ks / 4) * HALF_BYTES + (ks % 4) * 32, 0, 1024);
-          const uint64_t db = smem_desc_sw128(sdo + ks * 2048, HALF_BYTES, 1024);
-          umma_ss(tm_dv, da, db, idesc_acc, (it | ks) != 0);
-        }
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS_T; ++ks) {  // dK += dS^T Q
-          const uint64_t da = smem_desc_sw128(sdst + (ks / 4) * HALF_BYTES + (ks % 4) * 32, 0, 1024);
-          const uint64_t db = smem_desc_sw128(sq + ks * 2048, HALF_BYTES, 1024);
-          umma_ss(tm_dk, da, db, idesc_acc, (it | ks) != 0);
-        }
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS_T; ++ks) {  // dQ = dS K   (A = dS^T tile read MN-major)
-          const uint64_t da = smem_desc_sw128(sdst + ks * 2048, HALF_BYTES, 1024);
-          const uint64_t db = smem_desc_sw128(sk + ks * 2048, HALF_BYTES, 1024);
-          umma_ss(tm_dp, da, db, idesc_dq, ks != 0);
-        }
-        umma_commit(qdo_empty);
-        umma_commit(dq_full);
+        for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dK += dS^T Q
+          umma_ts(tm_dk, tm + 64 + ks * 8, smem_desc_sw128(sq + ks * 2048, QHALF_BYTES, 1024), idesc_acc,
+                  (it | ks) != 0);
+        umma_commit(&q_empty[s]);
       }
+      if (ok) umma_commit(acc_done);
     }
   } else {
-    // ------------------------------ compute warps ------------------------------
-    const int quarter = warp & 3;
-    const int r = quarter * 32 + lane;  // key row for S^T / dP^T, query row for dQ
+    // ------------------------------ compute warpgroups ------------------------------
+    const int wg = (warp - 2) >> 2;     // 0: even steps, 1: odd steps
+    const int quarter = warp & 3;       // TMEM lane quarter of this warp
+    const int r = quarter * 32 + lane;  // key row inside the tile == TMEM lane
     const int tid = r;
     const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
     const int kv_row = kv0 + r;
+    const uint32_t tm = tmem_base + wg * 128;
+    float* my_lse = s_lse + wg * BQ2;
+    float* my_delta = s_delta + wg * BQ2;
+    const int bar_id = 1 + wg;
     bool ok = true;
-    for (int it = 0; it < n_iter; ++it) {
+    for (int it = wg; it < n_iter; it += 2) {
       int li, hq, q0;
       decode_iter(it, li, hq, q0);
-      const uint32_t ph = it & 1;
-      // stage LSE and Delta of the 128 query columns (visible to every thread after the barrier)
-      {
+      // stage LSE (log2 domain) and Delta of the 64 query columns for this warpgroup
+      float l2 = 0.f, dl = 0.f;
+      if (tid < BQ2) {
         const int qc = q0 + tid;
         const size_t idx = (size_t(b) * p.Hq + hq) * p.S + qc;
-        const float l2 = qc < p.S ? p.lse[li][idx] * 1.4426950408889634f : INFINITY;
-        const float dl = qc < p.S ? p.delta[li][idx] : 0.f;
-        compute_bar_sync();  // previous iteration's readers are done with the staging arrays
-        s_lse[tid] = l2;
-        s_delta[tid] = dl;
-        compute_bar_sync();
+        l2 = qc < p.S ? p.lse[li][idx] * 1.4426950408889634f : INFINITY;
+        dl = qc < p.S ? p.delta[li][idx] : 0.f;
       }
-      ok = mbar_wait(st_full, ph, err);
+      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");  // previous step's readers are done
+      if (tid < BQ2) {
+        my_lse[tid] = l2;
+        my_delta[tid] = dl;
+      }
+      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+      ok = mbar_wait(&st_full[wg], (it >> 1) & 1, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc_fence_after_sync();
-      const bool diag = p.causal && (q0 < kv0 + BT);  // some (key, query) pairs of this tile are masked
-#pragma unroll 1
-      for (int c = 0; c < BT / 32; ++c) {
+      const bool diag = p.causal && (q0 < kv0 + BT);
+      uint32_t pk[32], dk[32];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
         uint32_t st[32], dp[32];
-        tmem_ld_x32(tm_st + lane_sel + c * 32, st);
-        tmem_ld_x32(tm_dp + lane_sel + c * 32, dp);
+        tmem_ld_x32(tm + lane_sel + c * 32, st);
+        tmem_ld_x32(tm + 64 + lane_sel + c * 32, dp);
         tmem_ld_wait();
-        uint32_t pt[16], ds[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
           float pv[2], dv[2];
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
             const int col = c * 32 + i + u;
-            float pr = fast_exp2(__uint_as_float(st[i + u]) * p.scale_log2 - s_lse[col]);
+            float pr = fast_exp2(fmaf(__uint_as_float(st[i + u]), p.scale_log2, -my_lse[col]));
             if (diag && (q0 + col < kv_row)) pr = 0.f;
-            if (kv_row >= p.S) pr = 0.f;
             pv[u] = pr;
-            dv[u] = pr * (__uint_as_float(dp[i + u]) - s_delta[col]);
+            dv[u] = pr * (__uint_as_float(dp[i + u]) - my_delta[col]);
           }
-          pt[i / 2] = pack_bf16(pv[0], pv[1]);
-          ds[i / 2] = pack_bf16(dv[0], dv[1]);
-        }
-#pragma unroll
-        for (int v4 = 0; v4 < 4; ++v4) {
-          const int chunk = c * 4 + v4;  // 16-byte chunk (8 query columns) of this key row
-          const uint32_t off = (chunk / 8) * HALF_BYTES + sw128_offset(r, chunk % 8);
-          *reinterpret_cast<uint4*>(smem + L::OFF_PT + off) =
-              make_uint4(pt[4 * v4], pt[4 * v4 + 1], pt[4 * v4 + 2], pt[4 * v4 + 3]);
-          *reinterpret_cast<uint4*>(smem + L::OFF_DST + off) =
-              make_uint4(ds[4 * v4], ds[4 * v4 + 1], ds[4 * v4 + 2], ds[4 * v4 + 3]);
+          pk[c * 16 + i / 2] = pack_bf16(pv[0], pv[1]);
+          dk[c * 16 + i / 2] = pack_bf16(dv[0], dv[1]);
         }
       }
-      fence_proxy_async_smem();
+      // keys beyond the sequence contribute nothing (their K/V rows are zero-filled; dK/dV rows are not stored)
+      tmem_st_x32(tm + lane_sel, pk);
+      tmem_st_x32(tm + 64 + lane_sel, dk);
+      tmem_st_wait();
       tc_fence_before_sync();
-      mbar_arrive(pds_ready);
-
-      ok = mbar_wait(dq_full, ph, err);
-      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-      tc_fence_after_sync();
-      {
-        const int q_row = q0 + r;
-        float* dst = p.dq_acc[li] + ((size_t(b) * p.S + q_row) * p.Hq + hq) * DH;
-#pragma unroll 1
-        for (int c = 0; c < DH / 32; ++c) {
-          uint32_t acc[32];
-          tmem_ld_x32(tm_dp + lane_sel + c * 32, acc);
-          tmem_ld_wait();
-          if (q_row < p.S) {
-#pragma unroll
-            for (int v4 = 0; v4 < 8; ++v4)
-              red_add_v4(dst + c * 32 + v4 * 4, __uint_as_float(acc[4 * v4]), __uint_as_float(acc[4 * v4 + 1]),
-                         __uint_as_float(acc[4 * v4 + 2]), __uint_as_float(acc[4 * v4 + 3]));
-          }
-        }
-      }
-      tc_fence_before_sync();
-      mbar_arrive(dq_free);
+      mbar_arrive(&pds_ready[wg]);
     }
-    if (ok && n_iter > 0) {
-      // dq_full of the last iteration also covers the last dV / dK MMAs
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      bool w = mbar_wait(acc_done, 0, err);
+      ok = __all_sync(0xffffffffu, w);
+    }
+    if (ok) {
       tc_fence_after_sync();
-      // tcgen05.ld is warp-collective: every lane loads, only rows inside the sequence store
+      // warpgroup 0 writes dK (scaled), warpgroup 1 writes dV; every lane loads, valid rows store
       const bool valid = kv_row < p.S;
       const size_t row_off = ((size_t(b) * p.S + (valid ? kv_row : 0)) * p.Hkv + hk) * DH;
-      float* dk = p.dk_sum + row_off;
-      float* dv = p.dv_sum + row_off;
+      float* dst = (wg == 0 ? p.dk_sum : p.dv_sum) + row_off;
+      const uint32_t src = (wg == 0 ? tm_dk : tm_dv) + lane_sel;
+      const float mul = wg == 0 ? p.scale : 1.f;
 #pragma unroll 1
       for (int c = 0; c < DH / 32; ++c) {
         uint32_t a[32];
-        tmem_ld_x32(tm_dk + lane_sel + c * 32, a);
+        tmem_ld_x32(src + c * 32, a);
         tmem_ld_wait();
         if (valid) {
 #pragma unroll
           for (int v4 = 0; v4 < 8; ++v4)
-            *reinterpret_cast<float4*>(dk + c * 32 + v4 * 4) =
-                make_float4(__uint_as_float(a[4 * v4]) * p.scale, __uint_as_float(a[4 * v4 + 1]) * p.scale,
-                            __uint_as_float(a[4 * v4 + 2]) * p.scale, __uint_as_float(a[4 * v4 + 3]) * p.scale);
+            *reinterpret_cast<float4*>(dst + c * 32 + v4 * 4) =
+                make_float4(__uint_as_float(a[4 * v4]) * mul, __uint_as_float(a[4 * v4 + 1]) * mul,
+                            __uint_as_float(a[4 * v4 + 2]) * mul, __uint_as_float(a[4 * v4 + 3]) * mul);
         }
-        tmem_ld_x32(tm_dv + lane_sel + c * 32, a);
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// =============================================================================================
+// dQ
+// =============================================================================================
+constexpr int DQ_THREADS = 192;  // warp 0 TMA, warp 1 MMA, warps 2-5 compute
+
+template <int DH>
+struct DqSmem {
+  static constexpr int TILE = BT * DH * 2;
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_DO = OFF_Q + TILE;
+  static constexpr int OFF_K = OFF_DO + TILE;      // [2]
+  static constexpr int OFF_V = OFF_K + 2 * TILE;   // [2]
+  static constexpr int OFF_BAR = OFF_V + 2 * TILE;
+  static constexpr int TOTAL = OFF_BAR + 256 + 1024;
+};
+
+struct DqParams {
+  CUtensorMap map_q, map_do, map_k, map_v;  // box rows 128
+  const float* lse;                         // [B,Hq,S]
+  const float* delta;                       // [B,Hq,S]
+  __nv_bfloat16* dq;                        // [B,S,Hq,dh]
+  int B, S, Hq, Hkv;
+  int causal;
+  float scale;
+  float scale_log2;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant__ DqParams p) {
+  using L = DqSmem<DH>;
+  constexpr int HALVES = DH / 64;
+  constexpr int KSTEPS_DH = DH / 16;
+  constexpr int KSTEPS_KV = BT / 16;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  uint64_t* qdo_full = bars + 0;
+  uint64_t* k_full = bars + 1;    // [2]
+  uint64_t* k_empty = bars + 3;   // [2]
+  uint64_t* v_full = bars + 5;    // [2]
+  uint64_t* v_empty = bars + 7;   // [2]
+  uint64_t* s_full = bars + 9;    // [2]
+  uint64_t* dp_full = bars + 11;
+  uint64_t* ds_ready = bars + 12; // 128 arrivals
+  uint64_t* dq_done = bars + 13;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  int* err = &g_bwd_status;
+
+  const int hq = blockIdx.x % p.Hq;
+  const int b = blockIdx.x / p.Hq;
+  const int n_qtiles = (p.S + BT - 1) / BT;
+  const int qt = n_qtiles - 1 - blockIdx.y;  // heaviest tiles first
+  const int hk = hq / (p.Hq / p.Hkv);
+  const int q0 = qt * BT;
+  const int kv_end = p.causal ? min(p.S, q0 + BT) : p.S;
+  const int n_kv = (kv_end + BT - 1) / BT;
+
+  if (threadIdx.x == 0) {
+    mbar_init(qdo_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1);
+      mbar_init(&k_empty[i], 1);
+      mbar_init(&v_full[i], 1);
+      mbar_init(&v_empty[i], 1);
+      mbar_init(&s_full[i], 1);
+    }
+    mbar_init(dp_full, 1);
+    mbar_init(ds_ready, 128);
+    mbar_init(dq_done, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tm_s = tmem_base;         // two score buffers of 128 columns
+  const uint32_t tm_dp = tmem_base + 256;  // dP, then dS (bf16) over its first 64 columns
+  const uint32_t tm_dq = tmem_base + 384;  // DH columns
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&p.map_q);
+      tma_prefetch_desc(&p.map_do);
+      tma_prefetch_desc(&p.map_k);
+      tma_prefetch_desc(&p.map_v);
+      mbar_expect_tx(qdo_full, 2 * L::TILE);
+#pragma unroll
+      for (int h = 0; h < HALVES; ++h) {
+        tma_load_4d(smem + L::OFF_Q + h * HALF_BYTES, &p.map_q, qdo_full, h * 64, hq, q0, b);
+        tma_load_4d(smem + L::OFF_DO + h * HALF_BYTES, &p.map_do, qdo_full, h * 64, hq, q0, b);
+      }
+      for (int j = 0; j < n_kv; ++j) {
+        const int s = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        if (!mbar_wait(&k_empty[s], ph ^ 1, err)) break;
+        mbar_expect_tx(&k_full[s], L::TILE);
+#pragma unroll
+        for (int h = 0; h < HALVES; ++h)
+          tma_load_4d(smem + L::OFF_K + s * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BT, b);
+        if (!mbar_wait(&v_empty[s], ph ^ 1, err)) break;
+        mbar_expect_tx(&v_full[s], L::TILE);
+#pragma unroll
+        for (int h = 0; h < HALVES; ++h)
+          tma_load_4d(smem + L::OFF_V + s * L::TILE + h * HALF_BYTES, &p.map_v, &v_full[s], h * 64, hk, j * BT, b);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = umma_idesc_bf16(BT, BT, 0, 0);
+      constexpr uint32_t idesc_dq = umma_idesc_bf16(BT, DH, 0, 1);  // A = dS from TMEM, B = K MN-major
+      const uint32_t sq = smem_u32(smem + L::OFF_Q), sdo = smem_u32(smem + L::OFF_DO);
+      bool ok = mbar_wait(qdo_full, 0, err);
+      auto issue_s = [&](int j) -> bool {
+        const int s = j & 1;
+        if (!mbar_wait(&k_full[s], (j >> 1) & 1, err)) return false;
+        tc_fence_after_sync();
+        const uint32_t sk = smem_u32(smem + L::OFF_K + s * L::TILE);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
+          const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
+          umma_ss(tm_s + s * BT, smem_desc_sw128(sq + off, 0, 1024), smem_desc_sw128(sk + off, 0, 1024), idesc_s,
+                  ks != 0);
+        }
+        umma_commit(&s_full[s]);
+        return true;
+      };
+      auto issue_dp = [&](int j) -> bool {
+        const int s = j & 1;
+        if (!mbar_wait(&v_full[s], (j >> 1) & 1, err)) return false;
+        tc_fence_after_sync();
+        const uint32_t sv = smem_u32(smem + L::OFF_V + s * L::TILE);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
+          const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
+          umma_ss(tm_dp, smem_desc_sw128(sdo + off, 0, 1024), smem_desc_sw128(sv + off, 0, 1024), idesc_s, ks != 0);
+        }
+        umma_commit(&v_empty[s]);
+        umma_commit(dp_full);
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      if (ok) ok = issue_dp(0);
+      for (int j = 0; j < n_kv && ok; ++j) {
+        // S_{j+1} goes to the other score buffer: its last readers finished before ds_ready(j-1)
+        if (j + 1 < n_kv && !issue_s(j + 1)) { ok = false; break; }
+        if (!mbar_wait(ds_ready, j & 1, err)) { ok = false; break; }
+        tc_fence_after_sync();
+        const int s = j & 1;
+        const uint32_t sk = smem_u32(smem + L::OFF_K + s * L::TILE);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ += dS K
+          umma_ts(tm_dq, tm_dp + ks * 8, smem_desc_sw128(sk + ks * 2048, HALF_BYTES, 1024), idesc_dq, (j | ks) != 0);
+        umma_commit(&k_empty[s]);
+        // dP_{j+1} overwrites the columns dS_j sits in: it follows dQ_j in the in-order tensor pipe
+        if (j + 1 < n_kv && !issue_dp(j + 1)) { ok = false; break; }
+      }
+      if (ok) umma_commit(dq_done);
+    }
+  } else {
+    // ------------------------------ compute warps ------------------------------
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;  // query row inside the tile == TMEM lane
+    const int q_row = q0 + r;
+    const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
+    const size_t stat_idx = (size_t(b) * p.Hq + hq) * p.S + (q_row < p.S ? q_row : 0);
+    const float lse2 = q_row < p.S ? p.lse[stat_idx] * 1.4426950408889634f : INFINITY;
+    const float dl = q_row < p.S ? p.delta[stat_idx] : 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kv; ++j) {
+      const int s = j & 1;
+      ok = mbar_wait(&s_full[s], (j >> 1) & 1, err);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      tc_fence_after_sync();
+      const int kvb = j * BT;
+      int lim = p.S - kvb;
+      if (p.causal) lim = min(lim, q_row - kvb + 1);
+      float pr[BT];
+#pragma unroll
+      for (int c = 0; c < BT / 32; ++c) {
+        uint32_t tmp[32];
+        tmem_ld_x32(tm_s + lane_sel + s * BT + c * 32, tmp);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float e = fast_exp2(fmaf(__uint_as_float(tmp[i]), p.scale_log2, -lse2));
+          pr[c * 32 + i] = (c * 32 + i < lim) ? e : 0.f;
+        }
+      }
+      ok = mbar_wait(dp_full, j & 1, err);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c = 0; c < BT / 32; ++c) {
+        uint32_t tmp[32];
+        tmem_ld_x32(tm_dp + lane_sel + c * 32, tmp);
+        tmem_ld_wait();
+        uint32_t ds[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float d0 = pr[c * 32 + 2 * i] * (__uint_as_float(tmp[2 * i]) - dl);
+          const float d1 = pr[c * 32 + 2 * i + 1] * (__uint_as_float(tmp[2 * i + 1]) - dl);
+          ds[i] = pack_bf16(d0, d1);
+        }
+        // dS (bf16 pairs) over dP's own columns: chunk c lands in columns [16c, 16c+16), already read
+        tmem_st_x16(tm_dp + lane_sel + c * 16, ds);
+      }
+      tmem_st_wait();
+      tc_fence_before_sync();
+      mbar_arrive(ds_ready);
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      bool w = mbar_wait(dq_done, 0, err);
+      ok = __all_sync(0xffffffffu, w);
+    }
+    if (ok) {
+      tc_fence_after_sync();
+      const bool valid = q_row < p.S;
+      __nv_bfloat16* dst = p.dq + ((size_t(b) * p.S + (valid ? q_row : 0)) * p.Hq + hq) * DH;
+#pragma unroll 1
+      for (int c = 0; c < DH / 32; ++c) {
+        uint32_t a[32];
+        tmem_ld_x32(tm_dq + lane_sel + c * 32, a);
         tmem_ld_wait();
         if (valid) {
 #pragma unroll
-          for (int v4 = 0; v4 < 8; ++v4)
-            *reinterpret_cast<float4*>(dv + c * 32 + v4 * 4) =
-                make_float4(__uint_as_float(a[4 * v4]), __uint_as_float(a[4 * v4 + 1]), __uint_as_float(a[4 * v4 + 2]),
-                            __uint_as_float(a[4 * v4 + 3]));
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(a[8 * v4 + 0]) * p.scale, __uint_as_float(a[8 * v4 + 1]) * p.scale);
+            v.y = pack_bf16(__uint_as_float(a[8 * v4 + 2]) * p.scale, __uint_as_float(a[8 * v4 + 3]) * p.scale);
+            v.z = pack_bf16(__uint_as_float(a[8 * v4 + 4]) * p.scale, __uint_as_float(a[8 * v4 + 5]) * p.scale);
+            v.w = pack_bf16(__uint_as_float(a[8 * v4 + 6]) * p.scale, __uint_as_float(a[8 * v4 + 7]) * p.scale);
+            *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = v;
+          }
         }
       }
     }
@@ -372,33 +613,14 @@ __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfl
   }
 }
 
-__global__ void dq_finish_kernel(const float4* __restrict__ acc, uint2* __restrict__ dq, size_t n4, float scale) {
-  const size_t stride = size_t(gridDim.x) * blockDim.x;
-  for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n4; i += stride) {
-    const float4 v = acc[i];
-    dq[i] = make_uint2(pack_bf16(v.x * scale, v.y * scale), pack_bf16(v.z * scale, v.w * scale));
-  }
-}
-
-int make_map_bshd(CUtensorMap* m, const void* base, int B, int S, int H, int dh) {
+int make_map_bshd(CUtensorMap* m, const void* base, int B, int S, int H, int dh, int rows) {
   uint64_t dims[4] = {uint64_t(dh), uint64_t(H), uint64_t(S), uint64_t(B)};
   uint64_t strides[3] = {uint64_t(dh) * 2, uint64_t(H) * dh * 2, uint64_t(S) * H * dh * 2};
-  uint32_t box[4] = {64, 1, BT, 1};
+  uint32_t box[4] = {64, 1, uint32_t(rows), 1};
   return make_tensor_map(m, base, 2, 4, dims, strides, box, true);
 }
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
-
-int max_group_size(int L, const int32_t* donor) {
-  int best = 0;
-  for (int d = 0; d < L; ++d) {
-    if (donor[d] != d) continue;
-    int n = 0;
-    for (int l = d; l < L; ++l) n += donor[l] == d;
-    best = n > best ? n : best;
-  }
-  return best;
-}
 
 }  // namespace
 
@@ -412,13 +634,10 @@ int attn_bwd_read_status() {
   return v;
 }
 
-// Workspace: Delta for the layers of one launch and the fp32 dQ accumulators of one launch.
+// Workspace: Delta [B,Hq,S] fp32 for every layer.
 size_t attn_bwd_workspace(const kvp_shape* s, const int32_t* donor) {
-  int g = max_group_size(s->L, donor);
-  if (g > MAX_GROUP) g = MAX_GROUP;
-  const size_t delta = align256(size_t(s->B) * s->Hq * s->S * 4);
-  const size_t dq = align256(size_t(s->B) * s->S * s->Hq * s->dh * 4);
-  return size_t(g) * (delta + dq);
+  (void)donor;
+  return size_t(s->L) * align256(size_t(s->B) * s->Hq * s->S * 4);
 }
 
 int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
@@ -429,57 +648,86 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
   const int dh = s->dh;
   const float sc = scale == 0.f ? 1.f / sqrtf(float(dh)) : scale;
   const size_t delta_bytes = align256(size_t(s->B) * s->Hq * s->S * 4);
-  const size_t dq_bytes = align256(size_t(s->B) * s->S * s->Hq * dh * 4);
-  const size_t n_q = size_t(s->B) * s->S * s->Hq * dh;
   uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
-  int gmax = max_group_size(s->L, donor);
-  if (gmax > MAX_GROUP) gmax = MAX_GROUP;
-  uint8_t* ws_delta = wsb;
-  uint8_t* ws_dq = wsb + size_t(gmax) * delta_bytes;
-  cudaError_t e;
-  if (dh == 128)
-    e = cudaFuncSetAttribute(attn_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::TOTAL);
-  else
-    e = cudaFuncSetAttribute(attn_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::TOTAL);
-  if (e != cudaSuccess) return KVP_ERR_CUDA;
+  cudaError_t e1, e2;
+  if (dh == 128) {
+    e1 = cudaFuncSetAttribute(dkdv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkdvSmem<128>::TOTAL);
+    e2 = cudaFuncSetAttribute(dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<128>::TOTAL);
+  } else {
+    e1 = cudaFuncSetAttribute(dkdv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkdvSmem<64>::TOTAL);
+    e2 = cudaFuncSetAttribute(dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<64>::TOTAL);
+  }
+  if (e1 != cudaSuccess || e2 != cudaSuccess) return KVP_ERR_CUDA;
 
+  // Delta for every layer
+  for (int l = 0; l < s->L; ++l) {
+    float* dl = reinterpret_cast<float*>(wsb + size_t(l) * delta_bytes);
+    const size_t rows = size_t(s->B) * s->S * s->Hq;
+    const int blocks = int(min(size_t(sm_count()) * 16, (rows + 7) / 8));
+    if (dh == 128)
+      delta_kernel<128><<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(o[l]),
+                                                    reinterpret_cast<const __nv_bfloat16*>(d_o[l]), dl, s->B, s->S,
+                                                    s->Hq);
+    else
+      delta_kernel<64><<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(o[l]),
+                                                   reinterpret_cast<const __nv_bfloat16*>(d_o[l]), dl, s->B, s->S,
+                                                   s->Hq);
+    note_launch();
+  }
+  if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
+
+  // dQ, one launch per layer
+  for (int l = 0; l < s->L; ++l) {
+    const int d = donor[l];
+    DqParams p;
+    int rc = make_map_bshd(&p.map_q, q[l], s->B, s->S, s->Hq, dh, BT);
+    if (rc == KVP_OK) rc = make_map_bshd(&p.map_do, d_o[l], s->B, s->S, s->Hq, dh, BT);
+    if (rc == KVP_OK) rc = make_map_bshd(&p.map_k, k[d], s->B, s->S, s->Hkv, dh, BT);
+    if (rc == KVP_OK) rc = make_map_bshd(&p.map_v, v[d], s->B, s->S, s->Hkv, dh, BT);
+    if (rc != KVP_OK) return rc;
+    p.lse = lse[l];
+    p.delta = reinterpret_cast<const float*>(wsb + size_t(l) * delta_bytes);
+    p.dq = reinterpret_cast<__nv_bfloat16*>(dq[l]);
+    p.B = s->B;
+    p.S = s->S;
+    p.Hq = s->Hq;
+    p.Hkv = s->Hkv;
+    p.causal = causal;
+    p.scale = sc;
+    p.scale_log2 = sc * 1.4426950408889634f;
+    dim3 grid(s->B * s->Hq, (s->S + BT - 1) / BT);
+    timing_before(KVP_KERNEL_ATTN_BWD_DQ, stream);
+    if (dh == 128)
+      dq_kernel<128><<<grid, DQ_THREADS, DqSmem<128>::TOTAL, stream>>>(p);
+    else
+      dq_kernel<64><<<grid, DQ_THREADS, DqSmem<64>::TOTAL, stream>>>(p);
+    timing_after(KVP_KERNEL_ATTN_BWD_DQ, stream);
+    note_launch();
+    if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
+  }
+
+  // dK / dV, one launch per donor group.  A launch writes (does not add to) the accumulators, so a
+  // donor shared by more than MAX_GROUP layers is not supported.
   for (int d = 0; d < s->L; ++d) {
     if (donor[d] != d) continue;
-    int members[64];
+    int members[MAX_GROUP];
     int n = 0;
     for (int l = d; l < s->L; ++l)
       if (donor[l] == d) {
-        if (n == MAX_GROUP) return KVP_ERR_UNSUPPORTED;  // more than MAX_GROUP layers share one donor
+        if (n == MAX_GROUP) return KVP_ERR_UNSUPPORTED;
         members[n++] = l;
       }
-    BwdParams p;
-    int rc = make_map_bshd(&p.map_k, k[d], s->B, s->S, s->Hkv, dh);
-    if (rc == KVP_OK) rc = make_map_bshd(&p.map_v, v[d], s->B, s->S, s->Hkv, dh);
+    DkdvParams p;
+    int rc = make_map_bshd(&p.map_k, k[d], s->B, s->S, s->Hkv, dh, BT);
+    if (rc == KVP_OK) rc = make_map_bshd(&p.map_v, v[d], s->B, s->S, s->Hkv, dh, BT);
     if (rc != KVP_OK) return rc;
-    if (cudaMemsetAsync(ws_dq, 0, size_t(n) * dq_bytes, stream) != cudaSuccess) return KVP_ERR_CUDA;
     for (int i = 0; i < MAX_GROUP; ++i) {
       const int l = members[i < n ? i : 0];
-      rc = make_map_bshd(&p.map_q[i], q[l], s->B, s->S, s->Hq, dh);
-      if (rc == KVP_OK) rc = make_map_bshd(&p.map_do[i], d_o[l], s->B, s->S, s->Hq, dh);
+      rc = make_map_bshd(&p.map_q[i], q[l], s->B, s->S, s->Hq, dh, BQ2);
+      if (rc == KVP_OK) rc = make_map_bshd(&p.map_do[i], d_o[l], s->B, s->S, s->Hq, dh, BQ2);
       if (rc != KVP_OK) return rc;
-      const int slot = i < n ? i : 0;
       p.lse[i] = lse[l];
-      p.delta[i] = reinterpret_cast<const float*>(ws_delta + size_t(slot) * delta_bytes);
-      p.dq_acc[i] = reinterpret_cast<float*>(ws_dq + size_t(slot) * dq_bytes);
-    }
-    for (int i = 0; i < n; ++i) {
-      const int l = members[i];
-      float* dl = reinterpret_cast<float*>(ws_delta + size_t(i) * delta_bytes);
-      const size_t rows = size_t(s->B) * s->S * s->Hq;
-      const int blocks = int(min(size_t(sm_count()) * 16, (rows + 7) / 8));
-      if (dh == 128)
-        delta_kernel<128><<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(o[l]),
-                                                      reinterpret_cast<const __nv_bfloat16*>(d_o[l]), dl, s->B, s->S,
-                                                      s->Hq);
-      else
-        delta_kernel<64><<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(o[l]),
-                                                     reinterpret_cast<const __nv_bfloat16*>(d_o[l]), dl, s->B, s->S,
-                                                     s->Hq);
+      p.delta[i] = reinterpret_cast<const float*>(wsb + size_t(l) * delta_bytes);
     }
     p.dk_sum = dk_sum[d];
     p.dv_sum = dv_sum[d];
@@ -494,19 +742,11 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     dim3 grid((s->S + BT - 1) / BT, s->Hkv, s->B);
     timing_before(KVP_KERNEL_ATTN_BWD, stream);
     if (dh == 128)
-      attn_bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::TOTAL, stream>>>(p);
+      dkdv_kernel<128><<<grid, DKDV_THREADS, DkdvSmem<128>::TOTAL, stream>>>(p);
     else
-      attn_bwd_kernel<64><<<grid, BWD_THREADS, BwdSmem<64>::TOTAL, stream>>>(p);
+      dkdv_kernel<64><<<grid, DKDV_THREADS, DkdvSmem<64>::TOTAL, stream>>>(p);
     timing_after(KVP_KERNEL_ATTN_BWD, stream);
-    note_launch(1 + 2 * n);  // main kernel, n delta pre-passes, n dQ finish passes
-    if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
-    for (int i = 0; i < n; ++i) {
-      const int l = members[i];
-      const size_t n4 = n_q / 4;
-      const int blocks = int(min(size_t(sm_count()) * 8, (n4 + 255) / 256));
-      dq_finish_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const float4*>(ws_dq + size_t(i) * dq_bytes),
-                                                   reinterpret_cast<uint2*>(dq[l]), n4, sc);
-    }
+    note_launch();
     if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
   }
   return KVP_OK;

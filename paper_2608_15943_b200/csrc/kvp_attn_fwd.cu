@@ -12,6 +12,10 @@
 // scores while the exponentials of the current tile are computed.
 #include <math.h>
 
+// P is handed to the P V product through TMEM (A operand from tensor memory) rather than through
+// shared memory.
+#define KVP_FWD_TS 1
+
 #include "kvp_host.h"
 #include "kvp_sm100.cuh"
 
@@ -173,9 +177,13 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         const uint32_t sv = smem_u32(smem + L::OFF_V + s * L::KV_BYTES);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_PV; ++ks) {
-          const uint64_t da = smem_desc_sw128(sp + (ks / 4) * HALF_BYTES + (ks % 4) * 32, 0, 1024);
           const uint64_t db = smem_desc_sw128(sv + ks * 2048, HALF_BYTES, 1024);
+#ifdef KVP_FWD_TS
+          umma_ts(tmem_o, tmem_s + s * BKV + ks * 8, db, idesc_pv, (j | ks) != 0);
+#else
+          const uint64_t da = smem_desc_sw128(sp + (ks / 4) * HALF_BYTES + (ks % 4) * 32, 0, 1024);
           umma_ss(tmem_o, da, db, idesc_pv, (j | ks) != 0);
+#endif
         }
         umma_commit(&v_empty[s]);
         umma_commit(pv_done);
@@ -230,6 +238,21 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         l_sum *= alpha;
         rescale = true;
       }
+#ifdef KVP_FWD_TS
+#pragma unroll
+      for (int c = 0; c < BKV / 64; ++c) {
+        uint32_t pk[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float e0 = fast_exp2(x[c * 64 + 2 * i] - m_used);
+          const float e1 = fast_exp2(x[c * 64 + 2 * i + 1] - m_used);
+          l_sum += e0 + e1;
+          pk[i] = pack_bf16(e0, e1);
+        }
+        tmem_st_x32(tmem_s + lane_sel + s * BKV + c * 32, pk);
+      }
+      tmem_st_wait();
+#else
       uint8_t* p_tile = smem + L::OFF_P + s * L::P_BYTES;
 #pragma unroll
       for (int c = 0; c < BKV / 8; ++c) {
@@ -247,6 +270,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         *reinterpret_cast<uint4*>(p_tile + (c / 8) * HALF_BYTES + sw128_offset(r, c % 8)) = v;
       }
       fence_proxy_async_smem();
+#endif
       if (j > 0) {
         // O may only be touched once P_{j-1} V_{j-1} has landed; this also protects the P buffer
         // that tile j+1 will overwrite.

@@ -43,7 +43,14 @@ int sm_count();
 
 // Bookkeeping for benchmarks: every kernel launch of the library is counted, and a caller may
 // ask for CUDA events to be recorded around the launches of one named kernel.
-enum { KVP_KERNEL_GEMM = 0, KVP_KERNEL_ATTN_FWD = 1, KVP_KERNEL_ATTN_BWD = 2, KVP_KERNEL_DECODE = 3, KVP_KERNEL_COUNT = 4 };
+enum {
+  KVP_KERNEL_GEMM = 0,
+  KVP_KERNEL_ATTN_FWD = 1,
+  KVP_KERNEL_ATTN_BWD = 2,     // dK/dV kernel
+  KVP_KERNEL_DECODE = 3,
+  KVP_KERNEL_ATTN_BWD_DQ = 4,  // dQ kernel
+  KVP_KERNEL_COUNT = 5
+};
 void note_launch(int n = 1);
 void timing_before(int kernel, cudaStream_t stream);
 void timing_after(int kernel, cudaStream_t stream);

@@ -176,27 +176,30 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     if (lane == 0) {
       constexpr uint32_t idesc_st = umma_idesc_bf16(BT, BQ2, 0, 0);   // [128 keys x 64 queries]
       constexpr uint32_t idesc_acc = umma_idesc_bf16(BT, DH, 0, 1);   // A from TMEM, B MN-major
-      const uint32_t sk = smem_u32(smem + L::OFF_K), sv = smem_u32(smem + L::OFF_V);
+      constexpr uint32_t hi = desc_hi_sw128(1024);
+      // low descriptor words of the resident tiles; per MMA only a constant is added
+      const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K), 0);
+      const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::OFF_V), 0);
+      const uint32_t ring = smem_u32(smem + L::OFF_RING);
       bool ok = mbar_wait(kv_full, 0, err);
       auto issue_scores = [&](int it) -> bool {
         const int s = it % DKDV_STAGES;
         if (!mbar_wait(&q_full[s], (it / DKDV_STAGES) & 1, err)) return false;
         tc_fence_after_sync();
-        const uint32_t sq = smem_u32(smem + L::OFF_RING + s * L::STAGE);
-        const uint32_t sdo = sq + L::Q_TILE;
+        const uint32_t q_lo = desc_lo_sw128(ring + s * L::STAGE, 0);
+        const uint32_t do_lo = desc_lo_sw128(ring + s * L::STAGE + L::Q_TILE, 0);
         const uint32_t tm = tmem_base + (it & 1) * 128;
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
           const uint32_t offb = (ks / 4) * QHALF_BYTES + (ks % 4) * 32;
-          umma_ss(tm, smem_desc_sw128(sk + offa, 0, 1024), smem_desc_sw128(sq + offb, 0, 1024), idesc_st, ks != 0);
+          umma_ss_w(tm, desc_lo_add(k_lo, offa), desc_lo_add(q_lo, offb), hi, idesc_st, ks != 0);
         }
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
           const uint32_t offb = (ks / 4) * QHALF_BYTES + (ks % 4) * 32;
-          umma_ss(tm + 64, smem_desc_sw128(sv + offa, 0, 1024), smem_desc_sw128(sdo + offb, 0, 1024), idesc_st,
-                  ks != 0);
+          umma_ss_w(tm + 64, desc_lo_add(v_lo, offa), desc_lo_add(do_lo, offb), hi, idesc_st, ks != 0);
         }
         umma_commit(&st_full[it & 1]);
         return true;
@@ -209,16 +212,15 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         if (!mbar_wait(&pds_ready[it & 1], (it >> 1) & 1, err)) { ok = false; break; }
         tc_fence_after_sync();
         const int s = it % DKDV_STAGES;
-        const uint32_t sq = smem_u32(smem + L::OFF_RING + s * L::STAGE);
-        const uint32_t sdo = sq + L::Q_TILE;
+        const uint32_t qmn_lo = desc_lo_sw128(ring + s * L::STAGE, QHALF_BYTES);                 // Q  as MN-major B
+        const uint32_t domn_lo = desc_lo_sw128(ring + s * L::STAGE + L::Q_TILE, QHALF_BYTES);    // dO as MN-major B
         const uint32_t tm = tmem_base + (it & 1) * 128;
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dV += P^T dO
-          umma_ts(tm_dv, tm + ks * 8, smem_desc_sw128(sdo + ks * 2048, QHALF_BYTES, 1024), idesc_acc, (it | ks) != 0);
+          umma_ts_w(tm_dv, tm + ks * 8, desc_lo_add(domn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dK += dS^T Q
-          umma_ts(tm_dk, tm + 64 + ks * 8, smem_desc_sw128(sq + ks * 2048, QHALF_BYTES, 1024), idesc_acc,
-                  (it | ks) != 0);
+          umma_ts_w(tm_dk, tm + 64 + ks * 8, desc_lo_add(qmn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0);
         umma_commit(&q_empty[s]);
       }
       if (ok) umma_commit(acc_done);
@@ -236,48 +238,68 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     float* my_delta = s_delta + wg * BQ2;
     const int bar_id = 1 + wg;
     bool ok = true;
+    // LSE (log2 domain) and Delta of a step's 64 query columns are fetched one step ahead, so their
+    // global-memory latency never sits between the score MMAs and the exponentials
+    auto load_stats = [&](int it_, float& l2_, float& dl_) {
+      l2_ = 0.f;
+      dl_ = 0.f;
+      if (tid < BQ2 && it_ < n_iter) {
+        int li_, hq_, q0_;
+        decode_iter(it_, li_, hq_, q0_);
+        const int qc = q0_ + tid;
+        const size_t idx = (size_t(b) * p.Hq + hq_) * p.S + (qc < p.S ? qc : 0);
+        l2_ = qc < p.S ? p.lse[li_][idx] * 1.4426950408889634f : INFINITY;
+        dl_ = qc < p.S ? p.delta[li_][idx] : 0.f;
+      }
+    };
+    float l2, dl;
+    load_stats(wg, l2, dl);
     for (int it = wg; it < n_iter; it += 2) {
       int li, hq, q0;
       decode_iter(it, li, hq, q0);
-      // stage LSE (log2 domain) and Delta of the 64 query columns for this warpgroup
-      float l2 = 0.f, dl = 0.f;
-      if (tid < BQ2) {
-        const int qc = q0 + tid;
-        const size_t idx = (size_t(b) * p.Hq + hq) * p.S + qc;
-        l2 = qc < p.S ? p.lse[li][idx] * 1.4426950408889634f : INFINITY;
-        dl = qc < p.S ? p.delta[li][idx] : 0.f;
-      }
       asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");  // previous step's readers are done
       if (tid < BQ2) {
         my_lse[tid] = l2;
         my_delta[tid] = dl;
       }
       asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+      load_stats(it + 2, l2, dl);
       ok = mbar_wait(&st_full[wg], (it >> 1) & 1, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc_fence_after_sync();
       const bool diag = p.causal && (q0 < kv0 + BT);
       uint32_t pk[32], dk[32];
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t st[32], dp[32];
-        tmem_ld_x32(tm + lane_sel + c * 32, st);
-        tmem_ld_x32(tm + 64 + lane_sel + c * 32, dp);
+      {
+        // all four TMEM loads are issued before the single wait, so their latencies overlap
+        uint32_t st0[32], st1[32], dp0[32], dp1[32];
+        tmem_ld_x32(tm + lane_sel, st0);
+        tmem_ld_x32(tm + 64 + lane_sel, dp0);
+        tmem_ld_x32(tm + lane_sel + 32, st1);
+        tmem_ld_x32(tm + 64 + lane_sel + 32, dp1);
         tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float pv[2], dv[2];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int col = c * 32 + i + u;
-            float pr = fast_exp2(fmaf(__uint_as_float(st[i + u]), p.scale_log2, -my_lse[col]));
-            if (diag && (q0 + col < kv_row)) pr = 0.f;
-            pv[u] = pr;
-            dv[u] = pr * (__uint_as_float(dp[i + u]) - my_delta[col]);
+        const int first_visible = diag ? kv_row - q0 : 0;  // query columns below this are masked for this key row
+        auto quad = [&](const uint32_t* st, const uint32_t* dp, int col, uint32_t* pk2, uint32_t* dk2) {
+          const float4 l4 = *reinterpret_cast<const float4*>(my_lse + col);
+          const float4 d4 = *reinterpret_cast<const float4*>(my_delta + col);
+          float e0 = fast_exp2(fmaf(__uint_as_float(st[0]), p.scale_log2, -l4.x));
+          float e1 = fast_exp2(fmaf(__uint_as_float(st[1]), p.scale_log2, -l4.y));
+          float e2 = fast_exp2(fmaf(__uint_as_float(st[2]), p.scale_log2, -l4.z));
+          float e3 = fast_exp2(fmaf(__uint_as_float(st[3]), p.scale_log2, -l4.w));
+          if (diag) {
+            e0 = col + 0 < first_visible ? 0.f : e0;
+            e1 = col + 1 < first_visible ? 0.f : e1;
+            e2 = col + 2 < first_visible ? 0.f : e2;
+            e3 = col + 3 < first_visible ? 0.f : e3;
           }
-          pk[c * 16 + i / 2] = pack_bf16(pv[0], pv[1]);
-          dk[c * 16 + i / 2] = pack_bf16(dv[0], dv[1]);
-        }
+          pk2[0] = pack_bf16(e0, e1);
+          pk2[1] = pack_bf16(e2, e3);
+          dk2[0] = pack_bf16(e0 * (__uint_as_float(dp[0]) - d4.x), e1 * (__uint_as_float(dp[1]) - d4.y));
+          dk2[1] = pack_bf16(e2 * (__uint_as_float(dp[2]) - d4.z), e3 * (__uint_as_float(dp[3]) - d4.w));
+        };
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) quad(st0 + i, dp0 + i, i, pk + i / 2, dk + i / 2);
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) quad(st1 + i, dp1 + i, 32 + i, pk + 16 + i / 2, dk + 16 + i / 2);
       }
       // keys beyond the sequence contribute nothing (their K/V rows are zero-filled; dK/dV rows are not stored)
       tmem_st_x32(tm + lane_sel, pk);
@@ -443,18 +465,20 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16(BT, BT, 0, 0);
       constexpr uint32_t idesc_dq = umma_idesc_bf16(BT, DH, 0, 1);  // A = dS from TMEM, B = K MN-major
-      const uint32_t sq = smem_u32(smem + L::OFF_Q), sdo = smem_u32(smem + L::OFF_DO);
+      constexpr uint32_t hi = desc_hi_sw128(1024);
+      const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q), 0);
+      const uint32_t do_lo = desc_lo_sw128(smem_u32(smem + L::OFF_DO), 0);
+      const uint32_t k_base = smem_u32(smem + L::OFF_K), v_base = smem_u32(smem + L::OFF_V);
       bool ok = mbar_wait(qdo_full, 0, err);
       auto issue_s = [&](int j) -> bool {
         const int s = j & 1;
         if (!mbar_wait(&k_full[s], (j >> 1) & 1, err)) return false;
         tc_fence_after_sync();
-        const uint32_t sk = smem_u32(smem + L::OFF_K + s * L::TILE);
+        const uint32_t k_lo = desc_lo_sw128(k_base + s * L::TILE, 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss(tm_s + s * BT, smem_desc_sw128(sq + off, 0, 1024), smem_desc_sw128(sk + off, 0, 1024), idesc_s,
-                  ks != 0);
+          umma_ss_w(tm_s + s * BT, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_s, ks != 0);
         }
         umma_commit(&s_full[s]);
         return true;
@@ -463,11 +487,11 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
         const int s = j & 1;
         if (!mbar_wait(&v_full[s], (j >> 1) & 1, err)) return false;
         tc_fence_after_sync();
-        const uint32_t sv = smem_u32(smem + L::OFF_V + s * L::TILE);
+        const uint32_t v_lo = desc_lo_sw128(v_base + s * L::TILE, 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss(tm_dp, smem_desc_sw128(sdo + off, 0, 1024), smem_desc_sw128(sv + off, 0, 1024), idesc_s, ks != 0);
+          umma_ss_w(tm_dp, desc_lo_add(do_lo, off), desc_lo_add(v_lo, off), hi, idesc_s, ks != 0);
         }
         umma_commit(&v_empty[s]);
         umma_commit(dp_full);
@@ -481,10 +505,10 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
         if (!mbar_wait(ds_ready, j & 1, err)) { ok = false; break; }
         tc_fence_after_sync();
         const int s = j & 1;
-        const uint32_t sk = smem_u32(smem + L::OFF_K + s * L::TILE);
+        const uint32_t kmn_lo = desc_lo_sw128(k_base + s * L::TILE, HALF_BYTES);  // K as MN-major B
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ += dS K
-          umma_ts(tm_dq, tm_dp + ks * 8, smem_desc_sw128(sk + ks * 2048, HALF_BYTES, 1024), idesc_dq, (j | ks) != 0);
+          umma_ts_w(tm_dq, tm_dp + ks * 8, desc_lo_add(kmn_lo, ks * 2048), hi, idesc_dq, (j | ks) != 0);
         umma_commit(&k_empty[s]);
         // dP_{j+1} overwrites the columns dS_j sits in: it follows dQ_j in the in-order tensor pipe
         if (j + 1 < n_kv && !issue_dp(j + 1)) { ok = false; break; }

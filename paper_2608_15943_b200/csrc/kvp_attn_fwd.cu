@@ -146,7 +146,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
     if (lane == 0) {
       constexpr uint32_t idesc_qk = umma_idesc_bf16(BQ, BKV, 0, 0);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(BQ, DH, 0, 1);
-      const uint32_t sq = smem_u32(smem + L::OFF_Q);
+      constexpr uint32_t hi = desc_hi_sw128(1024);
+      const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q), 0);
       bool ok = mbar_wait(q_full, 0, err);
       auto issue_qk = [&](int j) -> bool {
         const int s = j & 1;
@@ -154,12 +155,11 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         if (j >= 2 && !mbar_wait(&s_free[s], ph ^ 1, err)) return false;
         if (!mbar_wait(&k_full[s], ph, err)) return false;
         tc_fence_after_sync();
-        const uint32_t sk = smem_u32(smem + L::OFF_K + s * L::KV_BYTES);
+        const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K + s * L::KV_BYTES), 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_QK; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss(tmem_s + s * BKV, smem_desc_sw128(sq + off, 0, 1024), smem_desc_sw128(sk + off, 0, 1024), idesc_qk,
-                  ks != 0);
+          umma_ss_w(tmem_s + s * BKV, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0);
         }
         umma_commit(&k_empty[s]);
         umma_commit(&s_full[s]);
@@ -179,7 +179,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         for (int ks = 0; ks < KSTEPS_PV; ++ks) {
           const uint64_t db = smem_desc_sw128(sv + ks * 2048, HALF_BYTES, 1024);
 #ifdef KVP_FWD_TS
-          umma_ts(tmem_o, tmem_s + s * BKV + ks * 8, db, idesc_pv, (j | ks) != 0);
+          umma_ts_w(tmem_o, tmem_s + s * BKV + ks * 8, desc_lo_add(desc_lo_sw128(sv, HALF_BYTES), ks * 2048), hi,
+                    idesc_pv, (j | ks) != 0);
+          (void)db;
 #else
           const uint64_t da = smem_desc_sw128(sp + (ks / 4) * HALF_BYTES + (ks % 4) * 32, 0, 1024);
           umma_ss(tmem_o, da, db, idesc_pv, (j | ks) != 0);

@@ -349,14 +349,15 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
 // dQ
 // =============================================================================================
 constexpr int DQ_THREADS = 192;  // warp 0 TMA, warp 1 MMA, warps 2-5 compute
+constexpr int DQ_KSTAGES = 3;    // a K tile is read by S_j and again, a tile later, by dQ_j: keep three live
 
 template <int DH>
 struct DqSmem {
   static constexpr int TILE = BT * DH * 2;
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_DO = OFF_Q + TILE;
-  static constexpr int OFF_K = OFF_DO + TILE;      // [2]
-  static constexpr int OFF_V = OFF_K + 2 * TILE;   // [2]
+  static constexpr int OFF_K = OFF_DO + TILE;               // [DQ_KSTAGES]
+  static constexpr int OFF_V = OFF_K + DQ_KSTAGES * TILE;   // [2]
   static constexpr int OFF_BAR = OFF_V + 2 * TILE;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
@@ -383,15 +384,15 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* qdo_full = bars + 0;
-  uint64_t* k_full = bars + 1;    // [2]
-  uint64_t* k_empty = bars + 3;   // [2]
-  uint64_t* v_full = bars + 5;    // [2]
-  uint64_t* v_empty = bars + 7;   // [2]
-  uint64_t* s_full = bars + 9;    // [2]
-  uint64_t* dp_full = bars + 11;
-  uint64_t* ds_ready = bars + 12; // 128 arrivals
-  uint64_t* dq_done = bars + 13;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+  uint64_t* k_full = bars + 1;    // [DQ_KSTAGES]
+  uint64_t* k_empty = bars + 4;   // [DQ_KSTAGES]
+  uint64_t* v_full = bars + 7;    // [2]
+  uint64_t* v_empty = bars + 9;   // [2]
+  uint64_t* s_full = bars + 11;   // [2]
+  uint64_t* dp_full = bars + 13;
+  uint64_t* ds_ready = bars + 14; // 128 arrivals
+  uint64_t* dq_done = bars + 15;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -408,9 +409,11 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
 
   if (threadIdx.x == 0) {
     mbar_init(qdo_full, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < DQ_KSTAGES; ++i) {
       mbar_init(&k_full[i], 1);
       mbar_init(&k_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(&v_full[i], 1);
       mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1);
@@ -448,11 +451,12 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
       for (int j = 0; j < n_kv; ++j) {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
-        if (!mbar_wait(&k_empty[s], ph ^ 1, err)) break;
-        mbar_expect_tx(&k_full[s], L::TILE);
+        const int sk = j % DQ_KSTAGES;
+        if (!mbar_wait(&k_empty[sk], ((j / DQ_KSTAGES) & 1) ^ 1, err)) break;
+        mbar_expect_tx(&k_full[sk], L::TILE);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_K + s * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BT, b);
+          tma_load_4d(smem + L::OFF_K + sk * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[sk], h * 64, hk, j * BT, b);
         if (!mbar_wait(&v_empty[s], ph ^ 1, err)) break;
         mbar_expect_tx(&v_full[s], L::TILE);
 #pragma unroll
@@ -472,9 +476,10 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
       bool ok = mbar_wait(qdo_full, 0, err);
       auto issue_s = [&](int j) -> bool {
         const int s = j & 1;
-        if (!mbar_wait(&k_full[s], (j >> 1) & 1, err)) return false;
+        const int sk = j % DQ_KSTAGES;
+        if (!mbar_wait(&k_full[sk], (j / DQ_KSTAGES) & 1, err)) return false;
         tc_fence_after_sync();
-        const uint32_t k_lo = desc_lo_sw128(k_base + s * L::TILE, 0);
+        const uint32_t k_lo = desc_lo_sw128(k_base + sk * L::TILE, 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
@@ -504,7 +509,7 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
         if (j + 1 < n_kv && !issue_s(j + 1)) { ok = false; break; }
         if (!mbar_wait(ds_ready, j & 1, err)) { ok = false; break; }
         tc_fence_after_sync();
-        const int s = j & 1;
+        const int s = j % DQ_KSTAGES;
         const uint32_t kmn_lo = desc_lo_sw128(k_base + s * L::TILE, HALF_BYTES);  // K as MN-major B
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ += dS K

@@ -2,19 +2,16 @@
 // with its own queries to the keys/values of layer donor[l].
 //
 // One CTA owns a 128-row query tile of one (batch, query head) and walks the donor's K/V tiles.
-//   warp 0      TMA producer: Q once, then K_j / V_j into two-stage rings
+//   warp 0      TMA producer: Q once, then K_j / V_j into three-stage rings
 //   warp 1      tcgen05.mma issuer: S_j = Q K_j^T into one of two TMEM score buffers, and
-//               O += P_j V_j with P_j read from shared memory and V_j as an MN-major operand
+//               O += P_j V_j with P_j as the A operand FROM TMEM and V_j as an MN-major operand
 //   warps 2-5   online softmax, one thread per query row (TMEM lane == row, so the row maximum
-//               and sum need no cross-thread traffic); write P_j (bf16, 128-byte swizzle) to shared
-//               memory; rescale O in TMEM only when the running maximum moved by more than 2^8
+//               and sum need no cross-thread traffic); write P_j (bf16 pairs) back over the first
+//               64 columns of its score buffer; rescale O in TMEM only when the running maximum
+//               moved by more than 2^8
 // QK_{j+1} is issued before the softmax of tile j finishes, so the tensor pipe works on the next
 // scores while the exponentials of the current tile are computed.
 #include <math.h>
-
-// P is handed to the P V product through TMEM (A operand from tensor memory) rather than through
-// shared memory.
-#define KVP_FWD_TS 1
 
 #include "kvp_host.h"
 #include "kvp_sm100.cuh"
@@ -24,6 +21,7 @@ namespace {
 
 constexpr int BQ = 128, BKV = 128;
 constexpr int FWD_THREADS = 192;
+constexpr int FWD_STAGES = 3;  // K and V rings: deep enough to hide the TMA latency of a tile
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 __device__ int g_fwd_status;
@@ -32,12 +30,10 @@ template <int DH>
 struct FwdSmem {
   static constexpr int Q_BYTES = BQ * DH * 2;
   static constexpr int KV_BYTES = BKV * DH * 2;
-  static constexpr int P_BYTES = BQ * BKV * 2;
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + Q_BYTES;
-  static constexpr int OFF_V = OFF_K + 2 * KV_BYTES;
-  static constexpr int OFF_P = OFF_V + 2 * KV_BYTES;
-  static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
+  static constexpr int OFF_V = OFF_K + FWD_STAGES * KV_BYTES;
+  static constexpr int OFF_BAR = OFF_V + FWD_STAGES * KV_BYTES;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // + alignment slack
 };
 
@@ -68,15 +64,15 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* q_full = bars + 0;
-  uint64_t* k_full = bars + 1;    // [2]
-  uint64_t* k_empty = bars + 3;   // [2]
-  uint64_t* v_full = bars + 5;    // [2]
-  uint64_t* v_empty = bars + 7;   // [2]
-  uint64_t* s_full = bars + 9;    // [2]
-  uint64_t* s_free = bars + 11;   // [2]
-  uint64_t* p_ready = bars + 13;  // [2]
-  uint64_t* pv_done = bars + 15;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* k_full = bars + 1;     // [FWD_STAGES]
+  uint64_t* k_empty = bars + 4;    // [FWD_STAGES]
+  uint64_t* v_full = bars + 7;     // [FWD_STAGES]
+  uint64_t* v_empty = bars + 10;   // [FWD_STAGES]
+  uint64_t* s_full = bars + 13;    // [2]
+  uint64_t* s_free = bars + 15;    // [2]
+  uint64_t* p_ready = bars + 17;   // [2]
+  uint64_t* pv_done = bars + 19;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -93,11 +89,13 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < FWD_STAGES; ++i) {
       mbar_init(&k_full[i], 1);
       mbar_init(&k_empty[i], 1);
       mbar_init(&v_full[i], 1);
       mbar_init(&v_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1);
       mbar_init(&s_free[i], 128);
       mbar_init(&p_ready[i], 128);
@@ -127,8 +125,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
       for (int h = 0; h < HALVES; ++h) tma_load_4d(smem + L::OFF_Q + h * HALF_BYTES, &p.map_q, q_full, h * 64, hq, q0, b);
       bool ok = true;
       for (int j = 0; j < n_kv && ok; ++j) {
-        const int s = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
+        const int s = j % FWD_STAGES;
+        const uint32_t ph = (j / FWD_STAGES) & 1;
         if (!mbar_wait(&k_empty[s], ph ^ 1, err)) { ok = false; break; }
         mbar_expect_tx(&k_full[s], L::KV_BYTES);
 #pragma unroll
@@ -152,16 +150,17 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
       auto issue_qk = [&](int j) -> bool {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
+        const int st = j % FWD_STAGES;
         if (j >= 2 && !mbar_wait(&s_free[s], ph ^ 1, err)) return false;
-        if (!mbar_wait(&k_full[s], ph, err)) return false;
+        if (!mbar_wait(&k_full[st], (j / FWD_STAGES) & 1, err)) return false;
         tc_fence_after_sync();
-        const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K + s * L::KV_BYTES), 0);
+        const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K + st * L::KV_BYTES), 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_QK; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
           umma_ss_w(tmem_s + s * BKV, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0);
         }
-        umma_commit(&k_empty[s]);
+        umma_commit(&k_empty[st]);
         umma_commit(&s_full[s]);
         return true;
       };
@@ -170,24 +169,17 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         if (j + 1 < n_kv && !issue_qk(j + 1)) { ok = false; break; }
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
+        const int st = j % FWD_STAGES;
         if (!mbar_wait(&p_ready[s], ph, err)) { ok = false; break; }
-        if (!mbar_wait(&v_full[s], ph, err)) { ok = false; break; }
+        if (!mbar_wait(&v_full[st], (j / FWD_STAGES) & 1, err)) { ok = false; break; }
         tc_fence_after_sync();
-        const uint32_t sp = smem_u32(smem + L::OFF_P + s * L::P_BYTES);
-        const uint32_t sv = smem_u32(smem + L::OFF_V + s * L::KV_BYTES);
+        const uint32_t sv = smem_u32(smem + L::OFF_V + st * L::KV_BYTES);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_PV; ++ks) {
-          const uint64_t db = smem_desc_sw128(sv + ks * 2048, HALF_BYTES, 1024);
-#ifdef KVP_FWD_TS
           umma_ts_w(tmem_o, tmem_s + s * BKV + ks * 8, desc_lo_add(desc_lo_sw128(sv, HALF_BYTES), ks * 2048), hi,
                     idesc_pv, (j | ks) != 0);
-          (void)db;
-#else
-          const uint64_t da = smem_desc_sw128(sp + (ks / 4) * HALF_BYTES + (ks % 4) * 32, 0, 1024);
-          umma_ss(tmem_o, da, db, idesc_pv, (j | ks) != 0);
-#endif
         }
-        umma_commit(&v_empty[s]);
+        umma_commit(&v_empty[st]);
         umma_commit(pv_done);
       }
     }
@@ -240,7 +232,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         l_sum *= alpha;
         rescale = true;
       }
-#ifdef KVP_FWD_TS
 #pragma unroll
       for (int c = 0; c < BKV / 64; ++c) {
         uint32_t pk[32];
@@ -254,25 +245,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         tmem_st_x32(tmem_s + lane_sel + s * BKV + c * 32, pk);
       }
       tmem_st_wait();
-#else
-      uint8_t* p_tile = smem + L::OFF_P + s * L::P_BYTES;
-#pragma unroll
-      for (int c = 0; c < BKV / 8; ++c) {
-        float e[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          e[i] = fast_exp2(x[c * 8 + i] - m_used);
-          l_sum += e[i];
-        }
-        uint4 v;
-        v.x = pack_bf16(e[0], e[1]);
-        v.y = pack_bf16(e[2], e[3]);
-        v.z = pack_bf16(e[4], e[5]);
-        v.w = pack_bf16(e[6], e[7]);
-        *reinterpret_cast<uint4*>(p_tile + (c / 8) * HALF_BYTES + sw128_offset(r, c % 8)) = v;
-      }
-      fence_proxy_async_smem();
-#endif
       if (j > 0) {
         // O may only be touched once P_{j-1} V_{j-1} has landed; this also protects the P buffer
         // that tile j+1 will overwrite.

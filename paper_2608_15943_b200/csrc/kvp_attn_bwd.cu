@@ -538,17 +538,39 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
       const int kvb = j * BT;
       int lim = p.S - kvb;
       if (p.causal) lim = min(lim, q_row - kvb + 1);
-      float pr[BT];
+      // packed fp32x2 arithmetic throughout: P = exp2(S c - LSE), dS = P (dP - Delta)
+      const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
+      const uint64_t nl2 = pack_f2(-lse2, -lse2);
+      const uint64_t ndl2 = pack_f2(-dl, -dl);
+      uint64_t pr2[BT / 2];
+      {
+        const uint32_t ts = tm_s + lane_sel + s * BT;
+        uint32_t t0[32], t1[32], t2[32], t3[32];
+        tmem_ld_x32(ts, t0);
+        tmem_ld_x32(ts + 32, t1);
+        tmem_ld_wait();
+        tmem_ld_x32(ts + 64, t2);  // in flight while the first half is exponentiated
+        tmem_ld_x32(ts + 96, t3);
 #pragma unroll
-      for (int c = 0; c < BT / 32; ++c) {
-        uint32_t tmp[32];
-        tmem_ld_x32(tm_s + lane_sel + s * BT + c * 32, tmp);
+        for (int i = 0; i < 16; ++i) {
+          const uint64_t x0 = ffma2(pack_f2(__uint_as_float(t0[2 * i]), __uint_as_float(t0[2 * i + 1])), c2, nl2);
+          const uint64_t x1 = ffma2(pack_f2(__uint_as_float(t1[2 * i]), __uint_as_float(t1[2 * i + 1])), c2, nl2);
+          pr2[i] = pack_f2(fast_exp2(f2_lo(x0)), fast_exp2(f2_hi(x0)));
+          pr2[16 + i] = pack_f2(fast_exp2(f2_lo(x1)), fast_exp2(f2_hi(x1)));
+        }
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float e = fast_exp2(fmaf(__uint_as_float(tmp[i]), p.scale_log2, -lse2));
-          pr[c * 32 + i] = (c * 32 + i < lim) ? e : 0.f;
+        for (int i = 0; i < 16; ++i) {
+          const uint64_t x0 = ffma2(pack_f2(__uint_as_float(t2[2 * i]), __uint_as_float(t2[2 * i + 1])), c2, nl2);
+          const uint64_t x1 = ffma2(pack_f2(__uint_as_float(t3[2 * i]), __uint_as_float(t3[2 * i + 1])), c2, nl2);
+          pr2[32 + i] = pack_f2(fast_exp2(f2_lo(x0)), fast_exp2(f2_hi(x0)));
+          pr2[48 + i] = pack_f2(fast_exp2(f2_lo(x1)), fast_exp2(f2_hi(x1)));
         }
+      }
+      if (__any_sync(0xffffffffu, lim < BT)) {  // diagonal or ragged tile: zero the masked columns
+#pragma unroll
+        for (int i = 0; i < BT / 2; ++i)
+          pr2[i] = pack_f2(2 * i < lim ? f2_lo(pr2[i]) : 0.f, 2 * i + 1 < lim ? f2_hi(pr2[i]) : 0.f);
       }
       ok = mbar_wait(dp_full, j & 1, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
@@ -561,9 +583,9 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
         uint32_t ds[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const float d0 = pr[c * 32 + 2 * i] * (__uint_as_float(tmp[2 * i]) - dl);
-          const float d1 = pr[c * 32 + 2 * i + 1] * (__uint_as_float(tmp[2 * i + 1]) - dl);
-          ds[i] = pack_bf16(d0, d1);
+          const uint64_t d = fmul2(pr2[c * 16 + i],
+                                   fadd2(pack_f2(__uint_as_float(tmp[2 * i]), __uint_as_float(tmp[2 * i + 1])), ndl2));
+          ds[i] = pack_bf16(f2_lo(d), f2_hi(d));
         }
         // dS (bf16 pairs) over dP's own columns: chunk c lands in columns [16c, 16c+16), already read
         tmem_st_x16(tm_dp + lane_sel + c * 16, ds);

@@ -1,16 +1,16 @@
 // Causal GQA flash-attention forward over a donor map (Eq. 2-3 of the paper): layer l attends
 // with its own queries to the keys/values of layer donor[l].
 //
-// One CTA owns a 128-row query tile of one (batch, query head) and walks the donor's K/V tiles.
-//   warp 0      TMA producer: Q once, then K_j / V_j into three-stage rings
-//   warp 1      tcgen05.mma issuer: S_j = Q K_j^T into one of two TMEM score buffers, and
-//               O += P_j V_j with P_j as the A operand FROM TMEM and V_j as an MN-major operand
-//   warps 2-5   online softmax, one thread per query row (TMEM lane == row, so the row maximum
-//               and sum need no cross-thread traffic); write P_j (bf16 pairs) back over the first
-//               64 columns of its score buffer; rescale O in TMEM only when the running maximum
-//               moved by more than 2^8
-// QK_{j+1} is issued before the softmax of tile j finishes, so the tensor pipe works on the next
-// scores while the exponentials of the current tile are computed.
+// One CTA owns TWO adjacent 128-row query tiles (A, B) of one (batch, query head) and walks the
+// donor's K/V tiles once for both, so every K/V tile fetched by TMA feeds twice the tensor work.
+//   warp 0      TMA producer: Q_A, Q_B once, then K_j / V_j rings
+//   warp 1      tcgen05.mma issuer: S_X = Q_X K_j^T into tile X's 128 TMEM columns, and
+//               O_X += P_X V_j with P_X as the A operand FROM TMEM (bf16 pairs written back over the
+//               first 64 columns of S_X) and V_j as an MN-major B operand
+//   warps 2-5   softmax of tile A, warps 6-9 softmax of tile B: one thread per query row (TMEM lane
+//               == row, so the row maximum and sum need no cross-thread traffic), packed fp32x2
+//               arithmetic, O rescaled in TMEM only when the running maximum moved by more than 2^8
+// While one tile's exponentials run, the tensor pipe works on the other tile.
 #include <math.h>
 
 #include "kvp_host.h"
@@ -20,20 +20,22 @@ namespace kvp {
 namespace {
 
 constexpr int BQ = 128, BKV = 128;
-constexpr int FWD_THREADS = 192;
-constexpr int FWD_STAGES = 3;  // K and V rings: deep enough to hide the TMA latency of a tile
+constexpr int FWD_THREADS = 320;
+constexpr int FWD_KSTAGES = 3;
+constexpr int FWD_VSTAGES = 2;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr uint32_t HALF_BYTES = 128 * 128;  // one [128 rows x 128 B] block
 
 __device__ int g_fwd_status;
 
 template <int DH>
 struct FwdSmem {
-  static constexpr int Q_BYTES = BQ * DH * 2;
+  static constexpr int Q_BYTES = BQ * DH * 2;   // one query tile
   static constexpr int KV_BYTES = BKV * DH * 2;
-  static constexpr int OFF_Q = 0;
-  static constexpr int OFF_K = OFF_Q + Q_BYTES;
-  static constexpr int OFF_V = OFF_K + FWD_STAGES * KV_BYTES;
-  static constexpr int OFF_BAR = OFF_V + FWD_STAGES * KV_BYTES;
+  static constexpr int OFF_Q = 0;               // [2]
+  static constexpr int OFF_K = OFF_Q + 2 * Q_BYTES;
+  static constexpr int OFF_V = OFF_K + FWD_KSTAGES * KV_BYTES;
+  static constexpr int OFF_BAR = OFF_V + FWD_VSTAGES * KV_BYTES;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // + alignment slack
 };
 
@@ -58,21 +60,19 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
   constexpr int KSTEPS_QK = DH / 16;   // K dimension of S = Q K^T is dh
   constexpr int KSTEPS_PV = BKV / 16;  // K dimension of O = P V is the kv tile
   constexpr int HALVES = DH / 64;      // 64-column (128-byte) blocks per row of Q / K / V
-  constexpr uint32_t HALF_BYTES = 128 * 128;  // one [128 rows x 128 B] block
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* q_full = bars + 0;
-  uint64_t* k_full = bars + 1;     // [FWD_STAGES]
-  uint64_t* k_empty = bars + 4;    // [FWD_STAGES]
-  uint64_t* v_full = bars + 7;     // [FWD_STAGES]
-  uint64_t* v_empty = bars + 10;   // [FWD_STAGES]
-  uint64_t* s_full = bars + 13;    // [2]
-  uint64_t* s_free = bars + 15;    // [2]
-  uint64_t* p_ready = bars + 17;   // [2]
-  uint64_t* pv_done = bars + 19;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
+  uint64_t* k_full = bars + 1;                  // [KSTAGES]
+  uint64_t* k_empty = k_full + FWD_KSTAGES;     // [KSTAGES]
+  uint64_t* v_full = k_empty + FWD_KSTAGES;     // [VSTAGES]
+  uint64_t* v_empty = v_full + FWD_VSTAGES;     // [VSTAGES]
+  uint64_t* s_full = v_empty + FWD_VSTAGES;     // [2] per query tile
+  uint64_t* p_ready = s_full + 2;               // [2] per query tile (128 arrivals)
+  uint64_t* o_done = p_ready + 2;               // [2] per query tile
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 2);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -81,26 +81,35 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
   const int hq = blockIdx.x % p.Hq;
   const int b = blockIdx.x / p.Hq;
   const int n_qtiles = (p.S + BQ - 1) / BQ;
-  const int qt = n_qtiles - 1 - blockIdx.y;  // heaviest (deepest causal) tiles are dispatched first
+  const int n_pairs = (n_qtiles + 1) / 2;
+  const int pair = n_pairs - 1 - blockIdx.y;  // heaviest (deepest causal) pairs are dispatched first
   const int hk = hq / (p.Hq / p.Hkv);
-  const int q0 = qt * BQ;
-  const int kv_end = p.causal ? min(p.S, q0 + BQ) : p.S;
-  const int n_kv = (kv_end + BKV - 1) / BKV;
+  const int q0 = pair * 2 * BQ;               // first row of tile A; tile B starts at q0 + 128
+  // key tiles each query tile walks (tile B may not exist at a ragged end)
+  int n_kv[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    const int qs = q0 + x * BQ;
+    const int kv_end = p.causal ? min(p.S, qs + BQ) : p.S;
+    n_kv[x] = qs < p.S ? (kv_end + BKV - 1) / BKV : 0;
+  }
+  const int n_max = max(n_kv[0], n_kv[1]);
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int i = 0; i < FWD_STAGES; ++i) {
+    for (int i = 0; i < FWD_KSTAGES; ++i) {
       mbar_init(&k_full[i], 1);
       mbar_init(&k_empty[i], 1);
+    }
+    for (int i = 0; i < FWD_VSTAGES; ++i) {
       mbar_init(&v_full[i], 1);
       mbar_init(&v_empty[i], 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1);
-      mbar_init(&s_free[i], 128);
       mbar_init(&p_ready[i], 128);
+      mbar_init(&o_done[i], 1);
     }
-    mbar_init(pv_done, 1);
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -111,8 +120,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base;        // two score buffers of 128 columns
-  const uint32_t tmem_o = tmem_base + 256;  // DH columns
+  // tile X: scores / P at [X*128, X*128+128), output accumulator at [256 + X*128, ...)
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -120,23 +128,34 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
       tma_prefetch_desc(&p.map_q);
       tma_prefetch_desc(&p.map_k);
       tma_prefetch_desc(&p.map_v);
-      mbar_expect_tx(q_full, L::Q_BYTES);
+      mbar_expect_tx(q_full, 2 * L::Q_BYTES);  // rows beyond the sequence are zero-filled
 #pragma unroll
-      for (int h = 0; h < HALVES; ++h) tma_load_4d(smem + L::OFF_Q + h * HALF_BYTES, &p.map_q, q_full, h * 64, hq, q0, b);
-      bool ok = true;
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const int s = j % FWD_STAGES;
-        const uint32_t ph = (j / FWD_STAGES) & 1;
-        if (!mbar_wait(&k_empty[s], ph ^ 1, err)) { ok = false; break; }
+      for (int x = 0; x < 2; ++x)
+#pragma unroll
+        for (int h = 0; h < HALVES; ++h)
+          tma_load_4d(smem + L::OFF_Q + x * L::Q_BYTES + h * HALF_BYTES, &p.map_q, q_full, h * 64, hq, q0 + x * BQ, b);
+      auto load_k = [&](int j) -> bool {
+        const int s = j % FWD_KSTAGES;
+        if (!mbar_wait(&k_empty[s], ((j / FWD_KSTAGES) & 1) ^ 1, err)) return false;
         mbar_expect_tx(&k_full[s], L::KV_BYTES);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
           tma_load_4d(smem + L::OFF_K + s * L::KV_BYTES + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BKV, b);
-        if (!mbar_wait(&v_empty[s], ph ^ 1, err)) { ok = false; break; }
+        return true;
+      };
+      auto load_v = [&](int j) -> bool {
+        const int s = j % FWD_VSTAGES;
+        if (!mbar_wait(&v_empty[s], ((j / FWD_VSTAGES) & 1) ^ 1, err)) return false;
         mbar_expect_tx(&v_full[s], L::KV_BYTES);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
           tma_load_4d(smem + L::OFF_V + s * L::KV_BYTES + h * HALF_BYTES, &p.map_v, &v_full[s], h * 64, hk, j * BKV, b);
+        return true;
+      };
+      bool ok = n_max > 0 ? load_k(0) : true;
+      for (int j = 0; j < n_max && ok; ++j) {
+        if (j + 1 < n_max) ok = load_k(j + 1);  // scores run one tile ahead of the P V products
+        if (ok) ok = load_v(j);
       }
     }
   } else if (warp == 1) {
@@ -145,83 +164,93 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
       constexpr uint32_t idesc_qk = umma_idesc_bf16(BQ, BKV, 0, 0);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(BQ, DH, 0, 1);
       constexpr uint32_t hi = desc_hi_sw128(1024);
-      const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q), 0);
+      const uint32_t k_base = smem_u32(smem + L::OFF_K), v_base = smem_u32(smem + L::OFF_V);
       bool ok = mbar_wait(q_full, 0, err);
-      auto issue_qk = [&](int j) -> bool {
-        const int s = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        const int st = j % FWD_STAGES;
-        if (j >= 2 && !mbar_wait(&s_free[s], ph ^ 1, err)) return false;
-        if (!mbar_wait(&k_full[st], (j / FWD_STAGES) & 1, err)) return false;
-        tc_fence_after_sync();
-        const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K + st * L::KV_BYTES), 0);
+      auto issue_s = [&](int x, int j) {  // S_x(j) = Q_x K_j^T; K_j is known to be resident
+        const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q + x * L::Q_BYTES), 0);
+        const uint32_t k_lo = desc_lo_sw128(k_base + (j % FWD_KSTAGES) * L::KV_BYTES, 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_QK; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tmem_s + s * BKV, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0);
+          umma_ss_w(tmem_base + x * BKV, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0);
         }
-        umma_commit(&k_empty[st]);
-        umma_commit(&s_full[s]);
-        return true;
+        umma_commit(&s_full[x]);
       };
-      if (ok) ok = issue_qk(0);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        if (j + 1 < n_kv && !issue_qk(j + 1)) { ok = false; break; }
-        const int s = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        const int st = j % FWD_STAGES;
-        if (!mbar_wait(&p_ready[s], ph, err)) { ok = false; break; }
-        if (!mbar_wait(&v_full[st], (j / FWD_STAGES) & 1, err)) { ok = false; break; }
-        tc_fence_after_sync();
-        const uint32_t sv = smem_u32(smem + L::OFF_V + st * L::KV_BYTES);
+      auto issue_pv = [&](int x, int j) {  // O_x += P_x(j) V_j
+        const uint32_t v_lo = desc_lo_sw128(v_base + (j % FWD_VSTAGES) * L::KV_BYTES, HALF_BYTES);
 #pragma unroll
-        for (int ks = 0; ks < KSTEPS_PV; ++ks) {
-          umma_ts_w(tmem_o, tmem_s + s * BKV + ks * 8, desc_lo_add(desc_lo_sw128(sv, HALF_BYTES), ks * 2048), hi,
-                    idesc_pv, (j | ks) != 0);
+        for (int ks = 0; ks < KSTEPS_PV; ++ks)
+          umma_ts_w(tmem_base + 256 + x * 128, tmem_base + x * BKV + ks * 8, desc_lo_add(v_lo, ks * 2048), hi, idesc_pv,
+                    (j | ks) != 0);
+      };
+      if (ok && n_max > 0) {
+        ok = mbar_wait(&k_full[0], 0, err);
+        if (ok) {
+          tc_fence_after_sync();
+          if (n_kv[0] > 0) issue_s(0, 0);
+          if (n_kv[1] > 0) issue_s(1, 0);
+          umma_commit(&k_empty[0]);
         }
-        umma_commit(&v_empty[st]);
-        umma_commit(pv_done);
+      }
+      for (int j = 0; j < n_max && ok; ++j) {
+        const bool next = j + 1 < n_max;
+        if (next) {
+          if (!mbar_wait(&k_full[(j + 1) % FWD_KSTAGES], ((j + 1) / FWD_KSTAGES) & 1, err)) { ok = false; break; }
+        }
+        if (!mbar_wait(&v_full[j % FWD_VSTAGES], (j / FWD_VSTAGES) & 1, err)) { ok = false; break; }
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          if (j < n_kv[x]) {
+            if (!mbar_wait(&p_ready[x], j & 1, err)) { ok = false; break; }
+            tc_fence_after_sync();
+            issue_pv(x, j);
+            if (j + 1 == n_kv[x]) umma_commit(&o_done[x]);
+            // the score buffer of tile x is free again once P_x(j) V_j has been issued (in-order pipe)
+            if (j + 1 < n_kv[x]) issue_s(x, j + 1);
+          }
+        }
+        if (!ok) break;
+        umma_commit(&v_empty[j % FWD_VSTAGES]);
+        if (next) umma_commit(&k_empty[(j + 1) % FWD_KSTAGES]);
       }
     }
   } else {
     // ------------------------------ softmax + epilogue ------------------------------
+    const int x = (warp - 2) >> 2;      // query tile of this warpgroup
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;  // row inside the query tile == TMEM lane
-    const int q_row = q0 + r;
+    const int q_row = q0 + x * BQ + r;
     const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
+    const uint32_t tm_s = tmem_base + x * BKV + lane_sel;
+    const uint32_t tm_o = tmem_base + 256 + x * 128 + lane_sel;
+    const int my_n = n_kv[x];
+    const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
     float m_used = -INFINITY;  // running maximum (log2 domain) the exponentials are taken against
-    float l_sum = 0.f;
+    uint64_t l2 = 0ull;        // two partial row sums (packed lanes)
     bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      const int s = j & 1;
-      const uint32_t ph = (j >> 1) & 1;
-      ok = mbar_wait(&s_full[s], ph, err);
+    for (int j = 0; j < my_n; ++j) {
+      ok = mbar_wait(&s_full[x], j & 1, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc_fence_after_sync();
-      float x[BKV];
-#pragma unroll
-      for (int c = 0; c < BKV / 32; ++c) {
-        uint32_t tmp[32];
-        tmem_ld_x32(tmem_s + lane_sel + s * BKV + c * 32, tmp);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) x[c * 32 + i] = __uint_as_float(tmp[i]) * p.scale_log2;
-      }
-      tc_fence_before_sync();
-      mbar_arrive(&s_free[s]);
-
+      uint32_t sv[BKV];  // raw scores of this row
+      tmem_ld_x32(tm_s, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+      tmem_ld_x32(tm_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      tmem_ld_x32(tm_s + 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[64]));
+      tmem_ld_x32(tm_s + 96, *reinterpret_cast<uint32_t(*)[32]>(&sv[96]));
+      tmem_ld_wait();
       // columns of this tile visible to this row
       const int kv0 = j * BKV;
       int lim = p.S - kv0;
       if (p.causal) lim = min(lim, q_row - kv0 + 1);
-      if (lim < BKV) {
+      if (__any_sync(0xffffffffu, lim < BKV)) {
 #pragma unroll
         for (int i = 0; i < BKV; ++i)
-          if (i >= lim) x[i] = -INFINITY;
+          if (i >= lim) sv[i] = 0xff800000u;  // -inf
       }
-      float m_tile = x[0];
+      float m_raw = fmaxf(__uint_as_float(sv[0]), __uint_as_float(sv[1]));
 #pragma unroll
-      for (int i = 1; i < BKV; ++i) m_tile = fmaxf(m_tile, x[i]);
+      for (int i = 2; i < BKV; i += 2) m_raw = fmax3(m_raw, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+      const float m_tile = m_raw * p.scale_log2;  // the scale is positive, so the maximum commutes with it
       float alpha = 1.f;
       bool rescale = false;
       if (j == 0) {
@@ -229,57 +258,53 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
       } else if (m_tile > m_used + kRescaleThreshold) {
         alpha = fast_exp2(m_used - m_tile);
         m_used = m_tile;
-        l_sum *= alpha;
+        l2 = fmul2(l2, pack_f2(alpha, alpha));
         rescale = true;
       }
+      const uint64_t nm2 = pack_f2(-m_used, -m_used);
 #pragma unroll
-      for (int c = 0; c < BKV / 64; ++c) {
-        uint32_t pk[32];
+      for (int c = 0; c < BKV / 32; ++c) {
+        uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float e0 = fast_exp2(x[c * 64 + 2 * i] - m_used);
-          const float e1 = fast_exp2(x[c * 64 + 2 * i + 1] - m_used);
-          l_sum += e0 + e1;
+        for (int i = 0; i < 16; ++i) {
+          const uint64_t t = ffma2(pack_f2(__uint_as_float(sv[c * 32 + 2 * i]), __uint_as_float(sv[c * 32 + 2 * i + 1])), c2, nm2);
+          const float e0 = fast_exp2(f2_lo(t)), e1 = fast_exp2(f2_hi(t));
+          l2 = fadd2(l2, pack_f2(e0, e1));
           pk[i] = pack_bf16(e0, e1);
         }
-        tmem_st_x32(tmem_s + lane_sel + s * BKV + c * 32, pk);
+        tmem_st_x16(tm_s + c * 16, pk);  // P as bf16 pairs over the first 64 columns of the score buffer
+      }
+      // O_x is idle here: P_x(j-1) V_{j-1} precedes S_x(j) in the in-order tensor pipe
+      if (j > 0 && __any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+        for (int c = 0; c < DH / 32; ++c) {
+          uint32_t tmp[32];
+          tmem_ld_x32(tm_o + c * 32, tmp);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) tmp[i] = __float_as_uint(__uint_as_float(tmp[i]) * alpha);
+          tmem_st_x32(tm_o + c * 32, tmp);
+        }
       }
       tmem_st_wait();
-      if (j > 0) {
-        // O may only be touched once P_{j-1} V_{j-1} has landed; this also protects the P buffer
-        // that tile j+1 will overwrite.
-        ok = mbar_wait(pv_done, (j - 1) & 1, err);
-        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-        tc_fence_after_sync();
-        if (__any_sync(0xffffffffu, rescale)) {
-#pragma unroll
-          for (int c = 0; c < DH / 32; ++c) {
-            uint32_t tmp[32];
-            tmem_ld_x32(tmem_o + lane_sel + c * 32, tmp);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) tmp[i] = __float_as_uint(__uint_as_float(tmp[i]) * alpha);
-            tmem_st_x32(tmem_o + lane_sel + c * 32, tmp);
-          }
-          tmem_st_wait();
-        }
-        tc_fence_before_sync();
-      }
-      mbar_arrive(&p_ready[s]);
+      tc_fence_before_sync();
+      mbar_arrive(&p_ready[x]);
     }
-    if (ok) {
-      ok = mbar_wait(pv_done, (n_kv - 1) & 1, err);
-      ok = __all_sync(0xffffffffu, ok);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok && my_n > 0) {
+      bool w = mbar_wait(&o_done[x], 0, err);
+      ok = __all_sync(0xffffffffu, w);
     }
-    if (ok) {
+    if (ok && my_n > 0) {
       tc_fence_after_sync();
+      const float l_sum = f2_lo(l2) + f2_hi(l2);
       const float inv_l = 1.f / l_sum;
       const bool valid = q_row < p.S;
-      __nv_bfloat16* dst = p.o + ((size_t(b) * p.S + q_row) * p.Hq + hq) * DH;
+      __nv_bfloat16* dst = p.o + ((size_t(b) * p.S + (valid ? q_row : 0)) * p.Hq + hq) * DH;
 #pragma unroll
       for (int c = 0; c < DH / 32; ++c) {
         uint32_t tmp[32];
-        tmem_ld_x32(tmem_o + lane_sel + c * 32, tmp);
+        tmem_ld_x32(tm_o + c * 32, tmp);
         tmem_ld_wait();
         if (valid) {
 #pragma unroll
@@ -341,7 +366,8 @@ int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, c
   p.causal = causal;
   const float sc = scale == 0.f ? 1.f / sqrtf(float(s->dh)) : scale;
   p.scale_log2 = sc * 1.4426950408889634f;
-  dim3 grid(s->B * s->Hq, (s->S + BQ - 1) / BQ);
+  const int n_qtiles = (s->S + BQ - 1) / BQ;
+  dim3 grid(s->B * s->Hq, (n_qtiles + 1) / 2);
   cudaError_t e;
   timing_before(KVP_KERNEL_ATTN_FWD, stream);
   if (s->dh == 128) {

@@ -348,17 +348,17 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
 // =============================================================================================
 // dQ
 // =============================================================================================
-constexpr int DQ_THREADS = 192;  // warp 0 TMA, warp 1 MMA, warps 2-5 compute
-constexpr int DQ_KSTAGES = 3;    // a K tile is read by S_j and again, a tile later, by dQ_j: keep three live
+constexpr int DQ_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 query tile A, warps 6-9 query tile B
+constexpr int DQ_KSTAGES = 2;
 
 template <int DH>
 struct DqSmem {
   static constexpr int TILE = BT * DH * 2;
-  static constexpr int OFF_Q = 0;
-  static constexpr int OFF_DO = OFF_Q + TILE;
-  static constexpr int OFF_K = OFF_DO + TILE;               // [DQ_KSTAGES]
-  static constexpr int OFF_V = OFF_K + DQ_KSTAGES * TILE;   // [2]
-  static constexpr int OFF_BAR = OFF_V + 2 * TILE;
+  static constexpr int OFF_Q = 0;                          // [2] query tiles A, B
+  static constexpr int OFF_DO = OFF_Q + 2 * TILE;          // [2]
+  static constexpr int OFF_K = OFF_DO + 2 * TILE;          // [DQ_KSTAGES]
+  static constexpr int OFF_V = OFF_K + DQ_KSTAGES * TILE;  // one stage: V_j is only read by the two dP products
+  static constexpr int OFF_BAR = OFF_V + TILE;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
 
@@ -373,6 +373,11 @@ struct DqParams {
   float scale_log2;
 };
 
+// Two adjacent query tiles (A, B) share every K/V tile the CTA fetches.  Each query tile owns one
+// 128-column TMEM buffer that is reused through a key tile's life -- S (fp32) -> read by the tile's
+// warpgroup -> dP (fp32, same columns) -> read -> dS (bf16 pairs, first 64 columns) -> A operand of
+// dQ += dS K -- plus a DH-column dQ accumulator.  While one tile's exponentials run, the tensor pipe
+// works on the other tile.
 template <int DH>
 __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant__ DqParams p) {
   using L = DqSmem<DH>;
@@ -384,15 +389,16 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* qdo_full = bars + 0;
-  uint64_t* k_full = bars + 1;    // [DQ_KSTAGES]
-  uint64_t* k_empty = bars + 4;   // [DQ_KSTAGES]
-  uint64_t* v_full = bars + 7;    // [2]
-  uint64_t* v_empty = bars + 9;   // [2]
-  uint64_t* s_full = bars + 11;   // [2]
-  uint64_t* dp_full = bars + 13;
-  uint64_t* ds_ready = bars + 14; // 128 arrivals
-  uint64_t* dq_done = bars + 15;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* k_full = bars + 1;                 // [KSTAGES]
+  uint64_t* k_empty = k_full + DQ_KSTAGES;     // [KSTAGES]
+  uint64_t* v_full = k_empty + DQ_KSTAGES;
+  uint64_t* v_empty = v_full + 1;
+  uint64_t* s_full = v_empty + 1;              // [2] per query tile
+  uint64_t* s_read = s_full + 2;               // [2] S of the tile is in registers (128 arrivals)
+  uint64_t* dp_full = s_read + 2;              // [2]
+  uint64_t* ds_ready = dp_full + 2;            // [2] dS of the tile written (128 arrivals)
+  uint64_t* dq_done = ds_ready + 2;            // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dq_done + 2);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -401,11 +407,18 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
   const int hq = blockIdx.x % p.Hq;
   const int b = blockIdx.x / p.Hq;
   const int n_qtiles = (p.S + BT - 1) / BT;
-  const int qt = n_qtiles - 1 - blockIdx.y;  // heaviest tiles first
+  const int n_pairs = (n_qtiles + 1) / 2;
+  const int pair = n_pairs - 1 - blockIdx.y;  // heaviest pairs first
   const int hk = hq / (p.Hq / p.Hkv);
-  const int q0 = qt * BT;
-  const int kv_end = p.causal ? min(p.S, q0 + BT) : p.S;
-  const int n_kv = (kv_end + BT - 1) / BT;
+  const int q0 = pair * 2 * BT;
+  int n_kv[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    const int qs = q0 + x * BT;
+    const int kv_end = p.causal ? min(p.S, qs + BT) : p.S;
+    n_kv[x] = qs < p.S ? (kv_end + BT - 1) / BT : 0;
+  }
+  const int n_max = max(n_kv[0], n_kv[1]);
 
   if (threadIdx.x == 0) {
     mbar_init(qdo_full, 1);
@@ -413,14 +426,15 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
       mbar_init(&k_full[i], 1);
       mbar_init(&k_empty[i], 1);
     }
+    mbar_init(v_full, 1);
+    mbar_init(v_empty, 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&v_full[i], 1);
-      mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1);
+      mbar_init(&s_read[i], 128);
+      mbar_init(&dp_full[i], 1);
+      mbar_init(&ds_ready[i], 128);
+      mbar_init(&dq_done[i], 1);
     }
-    mbar_init(dp_full, 1);
-    mbar_init(ds_ready, 128);
-    mbar_init(dq_done, 1);
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -431,9 +445,7 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tm_s = tmem_base;         // two score buffers of 128 columns
-  const uint32_t tm_dp = tmem_base + 256;  // dP, then dS (bf16) over its first 64 columns
-  const uint32_t tm_dq = tmem_base + 384;  // DH columns
+  // query tile x: working buffer at [x*128, x*128+128), dQ accumulator at [256 + x*128, ...)
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -442,26 +454,35 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
       tma_prefetch_desc(&p.map_do);
       tma_prefetch_desc(&p.map_k);
       tma_prefetch_desc(&p.map_v);
-      mbar_expect_tx(qdo_full, 2 * L::TILE);
+      mbar_expect_tx(qdo_full, 4 * L::TILE);  // rows beyond the sequence are zero-filled
 #pragma unroll
-      for (int h = 0; h < HALVES; ++h) {
-        tma_load_4d(smem + L::OFF_Q + h * HALF_BYTES, &p.map_q, qdo_full, h * 64, hq, q0, b);
-        tma_load_4d(smem + L::OFF_DO + h * HALF_BYTES, &p.map_do, qdo_full, h * 64, hq, q0, b);
-      }
-      for (int j = 0; j < n_kv; ++j) {
-        const int s = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        const int sk = j % DQ_KSTAGES;
-        if (!mbar_wait(&k_empty[sk], ((j / DQ_KSTAGES) & 1) ^ 1, err)) break;
-        mbar_expect_tx(&k_full[sk], L::TILE);
+      for (int x = 0; x < 2; ++x)
 #pragma unroll
-        for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_K + sk * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[sk], h * 64, hk, j * BT, b);
-        if (!mbar_wait(&v_empty[s], ph ^ 1, err)) break;
-        mbar_expect_tx(&v_full[s], L::TILE);
+        for (int h = 0; h < HALVES; ++h) {
+          tma_load_4d(smem + L::OFF_Q + x * L::TILE + h * HALF_BYTES, &p.map_q, qdo_full, h * 64, hq, q0 + x * BT, b);
+          tma_load_4d(smem + L::OFF_DO + x * L::TILE + h * HALF_BYTES, &p.map_do, qdo_full, h * 64, hq, q0 + x * BT, b);
+        }
+      auto load_k = [&](int j) -> bool {
+        const int s = j % DQ_KSTAGES;
+        if (!mbar_wait(&k_empty[s], ((j / DQ_KSTAGES) & 1) ^ 1, err)) return false;
+        mbar_expect_tx(&k_full[s], L::TILE);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_V + s * L::TILE + h * HALF_BYTES, &p.map_v, &v_full[s], h * 64, hk, j * BT, b);
+          tma_load_4d(smem + L::OFF_K + s * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BT, b);
+        return true;
+      };
+      auto load_v = [&](int j) -> bool {
+        if (!mbar_wait(v_empty, (j & 1) ^ 1, err)) return false;
+        mbar_expect_tx(v_full, L::TILE);
+#pragma unroll
+        for (int h = 0; h < HALVES; ++h)
+          tma_load_4d(smem + L::OFF_V + h * HALF_BYTES, &p.map_v, v_full, h * 64, hk, j * BT, b);
+        return true;
+      };
+      bool ok = n_max > 0 ? load_k(0) : true;
+      for (int j = 0; j < n_max && ok; ++j) {
+        ok = load_v(j);
+        if (ok && j + 1 < n_max) ok = load_k(j + 1);
       }
     }
   } else if (warp == 1) {
@@ -470,143 +491,160 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
       constexpr uint32_t idesc_s = umma_idesc_bf16(BT, BT, 0, 0);
       constexpr uint32_t idesc_dq = umma_idesc_bf16(BT, DH, 0, 1);  // A = dS from TMEM, B = K MN-major
       constexpr uint32_t hi = desc_hi_sw128(1024);
-      const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q), 0);
-      const uint32_t do_lo = desc_lo_sw128(smem_u32(smem + L::OFF_DO), 0);
-      const uint32_t k_base = smem_u32(smem + L::OFF_K), v_base = smem_u32(smem + L::OFF_V);
+      const uint32_t k_base = smem_u32(smem + L::OFF_K);
+      const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::OFF_V), 0);
       bool ok = mbar_wait(qdo_full, 0, err);
-      auto issue_s = [&](int j) -> bool {
-        const int s = j & 1;
-        const int sk = j % DQ_KSTAGES;
-        if (!mbar_wait(&k_full[sk], (j / DQ_KSTAGES) & 1, err)) return false;
-        tc_fence_after_sync();
-        const uint32_t k_lo = desc_lo_sw128(k_base + sk * L::TILE, 0);
+      auto issue_s = [&](int x, int j) {  // S_x(j) = Q_x K_j^T
+        const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q + x * L::TILE), 0);
+        const uint32_t k_lo = desc_lo_sw128(k_base + (j % DQ_KSTAGES) * L::TILE, 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tm_s + s * BT, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_s, ks != 0);
+          umma_ss_w(tmem_base + x * BT, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_s, ks != 0);
         }
-        umma_commit(&s_full[s]);
-        return true;
+        umma_commit(&s_full[x]);
       };
-      auto issue_dp = [&](int j) -> bool {
-        const int s = j & 1;
-        if (!mbar_wait(&v_full[s], (j >> 1) & 1, err)) return false;
-        tc_fence_after_sync();
-        const uint32_t v_lo = desc_lo_sw128(v_base + s * L::TILE, 0);
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
-          const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tm_dp, desc_lo_add(do_lo, off), desc_lo_add(v_lo, off), hi, idesc_s, ks != 0);
+      if (ok && n_max > 0) {
+        ok = mbar_wait(&k_full[0], 0, err);
+        if (ok) {
+          tc_fence_after_sync();
+          if (n_kv[0] > 0) issue_s(0, 0);
+          if (n_kv[1] > 0) issue_s(1, 0);
         }
-        umma_commit(&v_empty[s]);
-        umma_commit(dp_full);
-        return true;
-      };
-      if (ok) ok = issue_s(0);
-      if (ok) ok = issue_dp(0);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        // S_{j+1} goes to the other score buffer: its last readers finished before ds_ready(j-1)
-        if (j + 1 < n_kv && !issue_s(j + 1)) { ok = false; break; }
-        if (!mbar_wait(ds_ready, j & 1, err)) { ok = false; break; }
-        tc_fence_after_sync();
-        const int s = j % DQ_KSTAGES;
-        const uint32_t kmn_lo = desc_lo_sw128(k_base + s * L::TILE, HALF_BYTES);  // K as MN-major B
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ += dS K
-          umma_ts_w(tm_dq, tm_dp + ks * 8, desc_lo_add(kmn_lo, ks * 2048), hi, idesc_dq, (j | ks) != 0);
-        umma_commit(&k_empty[s]);
-        // dP_{j+1} overwrites the columns dS_j sits in: it follows dQ_j in the in-order tensor pipe
-        if (j + 1 < n_kv && !issue_dp(j + 1)) { ok = false; break; }
       }
-      if (ok) umma_commit(dq_done);
+      for (int j = 0; j < n_max && ok; ++j) {
+        const uint32_t ph = j & 1;
+        if (!mbar_wait(v_full, ph, err)) { ok = false; break; }
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          if (j < n_kv[x]) {
+            // dP_x(j) overwrites S_x(j) once the warpgroup holds S_x(j) in registers
+            if (!mbar_wait(&s_read[x], ph, err)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t do_lo = desc_lo_sw128(smem_u32(smem + L::OFF_DO + x * L::TILE), 0);
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS_DH; ++ks) {
+              const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
+              umma_ss_w(tmem_base + x * BT, desc_lo_add(do_lo, off), desc_lo_add(v_lo, off), hi, idesc_s, ks != 0);
+            }
+            umma_commit(&dp_full[x]);
+          }
+        }
+        if (!ok) break;
+        umma_commit(v_empty);
+        const bool next = j + 1 < n_max;
+        if (next && !mbar_wait(&k_full[(j + 1) % DQ_KSTAGES], ((j + 1) / DQ_KSTAGES) & 1, err)) { ok = false; break; }
+        const uint32_t kmn_lo = desc_lo_sw128(k_base + (j % DQ_KSTAGES) * L::TILE, HALF_BYTES);  // K_j as MN-major B
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          if (j < n_kv[x]) {
+            if (!mbar_wait(&ds_ready[x], ph, err)) { ok = false; break; }
+            tc_fence_after_sync();
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ_x += dS_x(j) K_j
+              umma_ts_w(tmem_base + 256 + x * 128, tmem_base + x * BT + ks * 8, desc_lo_add(kmn_lo, ks * 2048), hi,
+                        idesc_dq, (j | ks) != 0);
+            if (j + 1 == n_kv[x]) umma_commit(&dq_done[x]);
+            // the tile's buffer takes the next scores right behind dQ_x(j) in the in-order tensor pipe
+            if (j + 1 < n_kv[x]) issue_s(x, j + 1);
+          }
+        }
+        if (!ok) break;
+        umma_commit(&k_empty[j % DQ_KSTAGES]);
+      }
     }
   } else {
-    // ------------------------------ compute warps ------------------------------
+    // ------------------------------ compute warpgroups ------------------------------
+    const int x = (warp - 2) >> 2;      // query tile of this warpgroup
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;  // query row inside the tile == TMEM lane
-    const int q_row = q0 + r;
+    const int q_row = q0 + x * BT + r;
     const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
+    const uint32_t tb = tmem_base + x * BT + lane_sel;
+    const int my_n = n_kv[x];
     const size_t stat_idx = (size_t(b) * p.Hq + hq) * p.S + (q_row < p.S ? q_row : 0);
     const float lse2 = q_row < p.S ? p.lse[stat_idx] * 1.4426950408889634f : INFINITY;
     const float dl = q_row < p.S ? p.delta[stat_idx] : 0.f;
+    const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
+    const uint64_t nl2 = pack_f2(-lse2, -lse2);
+    const uint64_t ndl2 = pack_f2(-dl, -dl);
     bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      const int s = j & 1;
-      ok = mbar_wait(&s_full[s], (j >> 1) & 1, err);
+    for (int j = 0; j < my_n; ++j) {
+      const uint32_t ph = j & 1;
+      ok = mbar_wait(&s_full[x], ph, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc_fence_after_sync();
       const int kvb = j * BT;
       int lim = p.S - kvb;
       if (p.causal) lim = min(lim, q_row - kvb + 1);
-      // packed fp32x2 arithmetic throughout: P = exp2(S c - LSE), dS = P (dP - Delta)
-      const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
-      const uint64_t nl2 = pack_f2(-lse2, -lse2);
-      const uint64_t ndl2 = pack_f2(-dl, -dl);
-      uint64_t pr2[BT / 2];
+      uint32_t pb[BT / 2];  // P as bf16 pairs, kept across the dP product
       {
-        const uint32_t ts = tm_s + lane_sel + s * BT;
         uint32_t t0[32], t1[32], t2[32], t3[32];
-        tmem_ld_x32(ts, t0);
-        tmem_ld_x32(ts + 32, t1);
+        tmem_ld_x32(tb, t0);
+        tmem_ld_x32(tb + 32, t1);
+        tmem_ld_x32(tb + 64, t2);
+        tmem_ld_x32(tb + 96, t3);
         tmem_ld_wait();
-        tmem_ld_x32(ts + 64, t2);  // in flight while the first half is exponentiated
-        tmem_ld_x32(ts + 96, t3);
+        tc_fence_before_sync();
+        mbar_arrive(&s_read[x]);  // the scores are in registers: dP may overwrite them
+        auto expo = [&](const uint32_t* t, uint32_t* out) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint64_t x0 = ffma2(pack_f2(__uint_as_float(t0[2 * i]), __uint_as_float(t0[2 * i + 1])), c2, nl2);
-          const uint64_t x1 = ffma2(pack_f2(__uint_as_float(t1[2 * i]), __uint_as_float(t1[2 * i + 1])), c2, nl2);
-          pr2[i] = pack_f2(fast_exp2(f2_lo(x0)), fast_exp2(f2_hi(x0)));
-          pr2[16 + i] = pack_f2(fast_exp2(f2_lo(x1)), fast_exp2(f2_hi(x1)));
-        }
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint64_t x0 = ffma2(pack_f2(__uint_as_float(t2[2 * i]), __uint_as_float(t2[2 * i + 1])), c2, nl2);
-          const uint64_t x1 = ffma2(pack_f2(__uint_as_float(t3[2 * i]), __uint_as_float(t3[2 * i + 1])), c2, nl2);
-          pr2[32 + i] = pack_f2(fast_exp2(f2_lo(x0)), fast_exp2(f2_hi(x0)));
-          pr2[48 + i] = pack_f2(fast_exp2(f2_lo(x1)), fast_exp2(f2_hi(x1)));
-        }
+          for (int i = 0; i < 16; ++i) {
+            const uint64_t v = ffma2(pack_f2(__uint_as_float(t[2 * i]), __uint_as_float(t[2 * i + 1])), c2, nl2);
+            out[i] = pack_bf16(fast_exp2(f2_lo(v)), fast_exp2(f2_hi(v)));
+          }
+        };
+        expo(t0, pb);
+        expo(t1, pb + 16);
+        expo(t2, pb + 32);
+        expo(t3, pb + 48);
       }
       if (__any_sync(0xffffffffu, lim < BT)) {  // diagonal or ragged tile: zero the masked columns
 #pragma unroll
-        for (int i = 0; i < BT / 2; ++i)
-          pr2[i] = pack_f2(2 * i < lim ? f2_lo(pr2[i]) : 0.f, 2 * i + 1 < lim ? f2_hi(pr2[i]) : 0.f);
+        for (int i = 0; i < BT / 2; ++i) {
+          uint32_t v = pb[i];
+          if (2 * i >= lim) v &= 0xffff0000u;
+          if (2 * i + 1 >= lim) v &= 0x0000ffffu;
+          pb[i] = v;
+        }
       }
-      ok = mbar_wait(dp_full, j & 1, err);
+      ok = mbar_wait(&dp_full[x], ph, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc_fence_after_sync();
 #pragma unroll
       for (int c = 0; c < BT / 32; ++c) {
         uint32_t tmp[32];
-        tmem_ld_x32(tm_dp + lane_sel + c * 32, tmp);
+        tmem_ld_x32(tb + c * 32, tmp);
         tmem_ld_wait();
         uint32_t ds[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const uint64_t d = fmul2(pr2[c * 16 + i],
-                                   fadd2(pack_f2(__uint_as_float(tmp[2 * i]), __uint_as_float(tmp[2 * i + 1])), ndl2));
+          const uint32_t pv = pb[c * 16 + i];
+          const uint64_t pf = pack_f2(__uint_as_float(pv << 16), __uint_as_float(pv & 0xffff0000u));
+          const uint64_t d = fmul2(pf, fadd2(pack_f2(__uint_as_float(tmp[2 * i]), __uint_as_float(tmp[2 * i + 1])), ndl2));
           ds[i] = pack_bf16(f2_lo(d), f2_hi(d));
         }
         // dS (bf16 pairs) over dP's own columns: chunk c lands in columns [16c, 16c+16), already read
-        tmem_st_x16(tm_dp + lane_sel + c * 16, ds);
+        tmem_st_x16(tb + c * 16, ds);
       }
       tmem_st_wait();
       tc_fence_before_sync();
-      mbar_arrive(ds_ready);
+      mbar_arrive(&ds_ready[x]);
     }
     ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
-      bool w = mbar_wait(dq_done, 0, err);
+    if (ok && my_n > 0) {
+      bool w = mbar_wait(&dq_done[x], 0, err);
       ok = __all_sync(0xffffffffu, w);
     }
-    if (ok) {
+    if (ok && my_n > 0) {
       tc_fence_after_sync();
       const bool valid = q_row < p.S;
       __nv_bfloat16* dst = p.dq + ((size_t(b) * p.S + (valid ? q_row : 0)) * p.Hq + hq) * DH;
+      const uint32_t src = tmem_base + 256 + x * 128 + lane_sel;
 #pragma unroll 1
       for (int c = 0; c < DH / 32; ++c) {
         uint32_t a[32];
-        tmem_ld_x32(tm_dq + lane_sel + c * 32, a);
+        tmem_ld_x32(src + c * 32, a);
         tmem_ld_wait();
         if (valid) {
 #pragma unroll
@@ -746,7 +784,7 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     p.causal = causal;
     p.scale = sc;
     p.scale_log2 = sc * 1.4426950408889634f;
-    dim3 grid(s->B * s->Hq, (s->S + BT - 1) / BT);
+    dim3 grid(s->B * s->Hq, ((s->S + BT - 1) / BT + 1) / 2);
     timing_before(KVP_KERNEL_ATTN_BWD_DQ, stream);
     if (dh == 128)
       dq_kernel<128><<<grid, DQ_THREADS, DqSmem<128>::TOTAL, stream>>>(p);

@@ -248,8 +248,8 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         decode_iter(it_, li_, hq_, q0_);
         const int qc = q0_ + tid;
         const size_t idx = (size_t(b) * p.Hq + hq_) * p.S + (qc < p.S ? qc : 0);
-        l2_ = qc < p.S ? p.lse[li_][idx] * 1.4426950408889634f : INFINITY;
-        dl_ = qc < p.S ? p.delta[li_][idx] : 0.f;
+        l2_ = qc < p.S ? -p.lse[li_][idx] * 1.4426950408889634f : -INFINITY;   // staged negated
+        dl_ = qc < p.S ? -p.delta[li_][idx] : 0.f;
       }
     };
     float l2, dl;
@@ -270,36 +270,47 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
       const bool diag = p.causal && (q0 < kv0 + BT);
       uint32_t pk[32], dk[32];
       {
-        // all four TMEM loads are issued before the single wait, so their latencies overlap
-        uint32_t st0[32], st1[32], dp0[32], dp1[32];
-        tmem_ld_x32(tm + lane_sel, st0);
-        tmem_ld_x32(tm + 64 + lane_sel, dp0);
-        tmem_ld_x32(tm + lane_sel + 32, st1);
-        tmem_ld_x32(tm + 64 + lane_sel + 32, dp1);
-        tmem_ld_wait();
+        // The staged statistics are stored negated (-LSE in the log2 domain, -Delta), so that the
+        // packed forms are plain fused multiply-adds: P = exp2(S c + (-LSE)), dS = P (dP + (-Delta)).
+        // Each half of the 64 columns: issue the TMEM loads, fetch the 32 + 32 statistics while they
+        // are in flight, then do the arithmetic on register data only.
+        const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
         const int first_visible = diag ? kv_row - q0 : 0;  // query columns below this are masked for this key row
-        auto quad = [&](const uint32_t* st, const uint32_t* dp, int col, uint32_t* pk2, uint32_t* dk2) {
-          const float4 l4 = *reinterpret_cast<const float4*>(my_lse + col);
-          const float4 d4 = *reinterpret_cast<const float4*>(my_delta + col);
-          float e0 = fast_exp2(fmaf(__uint_as_float(st[0]), p.scale_log2, -l4.x));
-          float e1 = fast_exp2(fmaf(__uint_as_float(st[1]), p.scale_log2, -l4.y));
-          float e2 = fast_exp2(fmaf(__uint_as_float(st[2]), p.scale_log2, -l4.z));
-          float e3 = fast_exp2(fmaf(__uint_as_float(st[3]), p.scale_log2, -l4.w));
-          if (diag) {
-            e0 = col + 0 < first_visible ? 0.f : e0;
-            e1 = col + 1 < first_visible ? 0.f : e1;
-            e2 = col + 2 < first_visible ? 0.f : e2;
-            e3 = col + 3 < first_visible ? 0.f : e3;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint32_t st[32], dp[32];
+          tmem_ld_x32(tm + lane_sel + h * 32, st);
+          tmem_ld_x32(tm + 64 + lane_sel + h * 32, dp);
+          ulonglong2 nl[8], nd[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            nl[i] = *reinterpret_cast<const ulonglong2*>(my_lse + h * 32 + i * 4);
+            nd[i] = *reinterpret_cast<const ulonglong2*>(my_delta + h * 32 + i * 4);
           }
-          pk2[0] = pack_bf16(e0, e1);
-          pk2[1] = pack_bf16(e2, e3);
-          dk2[0] = pack_bf16(e0 * (__uint_as_float(dp[0]) - d4.x), e1 * (__uint_as_float(dp[1]) - d4.y));
-          dk2[1] = pack_bf16(e2 * (__uint_as_float(dp[2]) - d4.z), e3 * (__uint_as_float(dp[3]) - d4.w));
-        };
+          tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) quad(st0 + i, dp0 + i, i, pk + i / 2, dk + i / 2);
-#pragma unroll
-        for (int i = 0; i < 32; i += 4) quad(st1 + i, dp1 + i, 32 + i, pk + 16 + i / 2, dk + 16 + i / 2);
+          for (int i = 0; i < 8; ++i) {
+            const uint64_t x0 = ffma2(pack_f2(__uint_as_float(st[4 * i]), __uint_as_float(st[4 * i + 1])), c2, nl[i].x);
+            const uint64_t x1 = ffma2(pack_f2(__uint_as_float(st[4 * i + 2]), __uint_as_float(st[4 * i + 3])), c2, nl[i].y);
+            float e0 = fast_exp2(f2_lo(x0)), e1 = fast_exp2(f2_hi(x0));
+            float e2 = fast_exp2(f2_lo(x1)), e3 = fast_exp2(f2_hi(x1));
+            if (diag) {
+              const int col = h * 32 + i * 4;
+              e0 = col + 0 < first_visible ? 0.f : e0;
+              e1 = col + 1 < first_visible ? 0.f : e1;
+              e2 = col + 2 < first_visible ? 0.f : e2;
+              e3 = col + 3 < first_visible ? 0.f : e3;
+            }
+            pk[h * 16 + 2 * i] = pack_bf16(e0, e1);
+            pk[h * 16 + 2 * i + 1] = pack_bf16(e2, e3);
+            const uint64_t d0 = fmul2(pack_f2(e0, e1),
+                                      fadd2(pack_f2(__uint_as_float(dp[4 * i]), __uint_as_float(dp[4 * i + 1])), nd[i].x));
+            const uint64_t d1 = fmul2(pack_f2(e2, e3),
+                                      fadd2(pack_f2(__uint_as_float(dp[4 * i + 2]), __uint_as_float(dp[4 * i + 3])), nd[i].y));
+            dk[h * 16 + 2 * i] = pack_bf16(f2_lo(d0), f2_hi(d0));
+            dk[h * 16 + 2 * i + 1] = pack_bf16(f2_lo(d1), f2_hi(d1));
+          }
+        }
       }
       // keys beyond the sequence contribute nothing (their K/V rows are zero-filled; dK/dV rows are not stored)
       tmem_st_x32(tm + lane_sel, pk);

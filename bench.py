@@ -35,6 +35,9 @@ from paper_2608_15943_b200 import workloads as W          # noqa: E402
 
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one-pass ncu captures of the
+# full-size launches, averaged over the launches of one step; summary and commands in profiles/traffic_full-size.md.
+NCU_TRAFFIC_BYTES = {"dkdv_kernel": 0.835e9, "dq_kernel": 0.662e9, "attn_fwd_kernel": 0.476e9, "decode_kernel": 77.96e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -358,7 +361,10 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
     top = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_step"])
     achieved = per_kernel[top]["algorithmic_tflops"]
     roofline = {"bound": "tensor", "kernel": top + "<128>", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None, "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
+                "frac": achieved / peak,
+                "traffic": None if args.small or cfg is not W.C2 else NCU_TRAFFIC_BYTES.get(top),
+                "traffic_unit": "bytes per launch (ncu, full-size capture)",
+                "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
                 "launches_per_step": per_kernel[top]["launches_per_step"],
                 "kernel_ms_per_step": per_kernel[top]["ms_per_step"],
                 "share_of_step": per_kernel[top]["share_of_step"],
@@ -449,7 +455,10 @@ def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, st
         "e2e": {"value": world * cfg.B / (ms_e2e / e2e_steps * 1e-3), "unit": "tokens/s",
                 "h2d_bytes_per_step": runner.h2d, "d2h_bytes_per_step": runner.d2h},
         "roofline": {"bound": "hbm", "kernel": "decode_kernel<128>", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "peak_kind": f"{peaks_kind} copy bandwidth",
+                     "frac": achieved / peak,
+                     "traffic": None if args.small else NCU_TRAFFIC_BYTES["decode_kernel"],
+                     "traffic_unit": "bytes per launch (ncu, full-size capture)",
+                     "algorithmic_bytes_per_launch": step_bytes, "peak_kind": f"{peaks_kind} copy bandwidth",
                      "kernel_ms_per_step": k_ms, "share_of_step": k_ms / ms_step,
                      "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
         "device_status": kvp.status_string(kvp.device_status()),

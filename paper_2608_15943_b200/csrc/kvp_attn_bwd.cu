@@ -6,11 +6,13 @@
 //               consumer layers, the Hq/Hkv query heads of the KV head's group, and every 64-row query
 //               tile the causal mask lets see the keys.  dK and dV of the donor are therefore summed on
 //               chip across layers and heads and written to HBM once.  Per step, transposed so that TMEM
-//               lane == key row:  S^T = K Q^T, dP^T = V dO^T (tcgen05, operands in shared memory);
-//               P^T = exp2(S^T c - LSE), dS^T = P^T (dP^T - Delta) are written back as bf16 over the
-//               same TMEM columns and fed to dV += P^T dO, dK += dS^T Q as the A operand FROM TMEM --
-//               P and dS never touch shared memory.  Two TMEM buffer sets and two compute warpgroups
-//               alternate, so the tensor pipe works on step n+1 while step n's exponentials run.
+//               lane == key row:  S^T = K Q^T, dP^T = V dO^T (tcgen05, operands in shared memory), each
+//               followed by one rank-3 MMA that subtracts the query's LSE/scale resp. Delta (a bf16
+//               three-term split against a tile of ones), so the accumulators already hold the
+//               exponent and dP - Delta; P^T = exp2(c acc), dS^T = P^T acc' are written back as bf16
+//               over the same TMEM columns and fed to dV += P^T dO, dK += dS^T Q as the A operand FROM
+//               TMEM -- P and dS never touch shared memory.  Two TMEM buffer sets alternate between
+//               steps; both compute warpgroups work on every step, each on half of its query columns.
 //
 //  dq_kernel    Q-stationary (like the forward).  One CTA owns a 128-row query tile of one (layer,
 //               batch, query head) and walks the donor's K/V tiles: S = Q K^T, dP = dO V^T,
@@ -57,9 +59,9 @@ struct DkdvSmem {
   static constexpr int OFF_K = 0;
   static constexpr int OFF_V = OFF_K + KV_TILE;
   static constexpr int OFF_RING = OFF_V + KV_TILE;
-  static constexpr int OFF_LSE = OFF_RING + DKDV_STAGES * STAGE;  // [2][64] floats
-  static constexpr int OFF_DELTA = OFF_LSE + 2 * BQ2 * 4;
-  static constexpr int OFF_BAR = OFF_DELTA + 2 * BQ2 * 4;
+  static constexpr int OFF_ONES = OFF_RING + DKDV_STAGES * STAGE;  // [128 x 16] bf16, unswizzled K-major
+  static constexpr int OFF_STAT = OFF_ONES + 4096;                 // [2 sets][lse, delta][64 x 16] bf16
+  static constexpr int OFF_BAR = OFF_STAT + 4 * 2048;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
 
@@ -78,6 +80,31 @@ struct DkdvParams {
   float scale_log2;
 };
 
+// Unswizzled K-major operand tile of 16 bf16 per row: two halves of 8 columns, each half stored as
+// rows of 16 bytes (8 rows = one 128-byte core matrix).  SBO = 128, LBO = rows * 16.
+__host__ __device__ constexpr uint32_t desc_hi_plain(uint32_t sbo_bytes) { return ((sbo_bytes >> 4) & 0x3FFF) | (1u << 14); }
+__device__ __forceinline__ uint32_t desc_lo_plain(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFF) >> 4) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
+}
+// v = h + m + l with h, m, l bf16: 24 significant bits, so a bf16 MMA can add v exactly enough
+__device__ __forceinline__ uint4 split3_bf16(float v) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(h);
+  const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+  const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
+  uint4 out;
+  out.x = uint32_t(__bfloat16_as_ushort(h)) | (uint32_t(__bfloat16_as_ushort(m)) << 16);
+  out.y = uint32_t(__bfloat16_as_ushort(l));
+  out.z = 0u;
+  out.w = 0u;
+  return out;
+}
+
+// Per 64-query step, transposed so that TMEM lane == key row: S^T = K Q^T and dP^T = V dO^T.  The
+// per-query statistics are applied BY THE TENSOR CORE: one extra K-step multiplies a [128 x 16] tile
+// of ones (first three columns) with a [64 x 16] tile holding -LSE/scale (resp. -Delta) of each query
+// split into three bf16 terms, so the accumulators already hold S - LSE/scale and dP - Delta and the
+// threads need no per-column operand: P^T = exp2(c * acc), dS^T = P^T * acc'.
 template <int DH>
 __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_constant__ DkdvParams p) {
   using L = DkdvSmem<DH>;
@@ -92,11 +119,10 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
   uint64_t* q_full = bars + 1;                    // [STAGES]
   uint64_t* q_empty = q_full + DKDV_STAGES;       // [STAGES]
   uint64_t* st_full = q_empty + DKDV_STAGES;      // [2]  S^T and dP^T of buffer set b are in TMEM
-  uint64_t* pds_ready = st_full + 2;              // [2]  P^T and dS^T of buffer set b written (128 arrivals)
-  uint64_t* acc_done = pds_ready + 2;             // all MMAs have completed
+  uint64_t* pds_ready = st_full + 2;              // [2]  P^T, dS^T written and the set's next statistics staged
+  uint64_t* stat0 = pds_ready + 2;                // statistics of the first two steps staged (256 arrivals)
+  uint64_t* acc_done = stat0 + 1;                 // all MMAs have completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
-  float* s_lse = reinterpret_cast<float*>(smem + L::OFF_LSE);      // [2][64]
-  float* s_delta = reinterpret_cast<float*>(smem + L::OFF_DELTA);  // [2][64]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -120,11 +146,19 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&st_full[i], 1);
-      mbar_init(&pds_ready[i], 128);
+      mbar_init(&pds_ready[i], 256);
     }
+    mbar_init(stat0, 256);
     mbar_init(acc_done, 1);
     mbar_fence_init();
   }
+  // constant operand tiles: ones in the first three columns; statistics tiles start as zeros
+  for (int i = threadIdx.x; i < (4096 + 4 * 2048) / 16; i += blockDim.x) {
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (i < 128) v = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);  // row i, columns 0-7 = 1,1,1,0,0,0,0,0
+    *reinterpret_cast<uint4*>(smem + L::OFF_ONES + i * 16) = v;
+  }
+  fence_proxy_async_smem();
   if (warp == 1) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
@@ -173,15 +207,20 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
       constexpr uint32_t idesc_st = umma_idesc_bf16(BT, BQ2, 0, 0);   // [128 keys x 64 queries]
       constexpr uint32_t idesc_acc = umma_idesc_bf16(BT, DH, 0, 1);   // A from TMEM, B MN-major
       constexpr uint32_t hi = desc_hi_sw128(1024);
+      constexpr uint32_t hi_plain = desc_hi_plain(128);
       // low descriptor words of the resident tiles; per MMA only a constant is added
       const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K), 0);
       const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::OFF_V), 0);
+      const uint32_t ones_lo = desc_lo_plain(smem_u32(smem + L::OFF_ONES), 2048);
+      const uint32_t stat_base = smem_u32(smem + L::OFF_STAT);
       const uint32_t ring = smem_u32(smem + L::OFF_RING);
       bool ok = mbar_wait(kv_full, 0, err);
+      if (ok) ok = mbar_wait(stat0, 0, err);
       auto issue_scores = [&](int it) -> bool {
         const int s = it % DKDV_STAGES;
         if (!mbar_wait(&q_full[s], (it / DKDV_STAGES) & 1, err)) return false;
@@ -189,25 +228,29 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         const uint32_t q_lo = desc_lo_sw128(ring + s * L::STAGE, 0);
         const uint32_t do_lo = desc_lo_sw128(ring + s * L::STAGE + L::Q_TILE, 0);
         const uint32_t tm = tmem_base + (it & 1) * 128;
+        const uint32_t stat_lo = desc_lo_plain(stat_base + (it & 1) * 4096, 1024);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
           const uint32_t offb = (ks / 4) * QHALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tm, desc_lo_add(k_lo, offa), desc_lo_add(q_lo, offb), hi, idesc_st, ks != 0);
+          umma_ss_w(tm, desc_lo_add(k_lo, offa), desc_lo_add(q_lo, offb), hi, idesc_st, ks != 0, leader);
         }
+        umma_ss_w(tm, ones_lo, stat_lo, hi_plain, idesc_st, 1, leader);                          // S^T -= LSE / scale
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
           const uint32_t offb = (ks / 4) * QHALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tm + 64, desc_lo_add(v_lo, offa), desc_lo_add(do_lo, offb), hi, idesc_st, ks != 0);
+          umma_ss_w(tm + 64, desc_lo_add(v_lo, offa), desc_lo_add(do_lo, offb), hi, idesc_st, ks != 0, leader);
         }
-        umma_commit(&st_full[it & 1]);
+        umma_ss_w(tm + 64, ones_lo, desc_lo_add(stat_lo, 2048), hi_plain, idesc_st, 1, leader);  // dP^T -= Delta
+        umma_commit(&st_full[it & 1], leader);
         return true;
       };
       if (ok && n_iter > 0) ok = issue_scores(0);
       for (int it = 0; it < n_iter && ok; ++it) {
         // scores of the next step go to the other buffer set; its previous readers (the accumulate
-        // MMAs of step it-1) precede this in the in-order tensor pipe
+        // MMAs of step it-1) precede this in the in-order tensor pipe, and its statistics tile was
+        // staged before pds_ready(it-1)
         if (it + 1 < n_iter && !issue_scores(it + 1)) { ok = false; break; }
         if (!mbar_wait(&pds_ready[it & 1], (it >> 1) & 1, err)) { ok = false; break; }
         tc_fence_after_sync();
@@ -217,107 +260,102 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         const uint32_t tm = tmem_base + (it & 1) * 128;
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dV += P^T dO
-          umma_ts_w(tm_dv, tm + ks * 8, desc_lo_add(domn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0);
+          umma_ts_w(tm_dv, tm + ks * 8 + (ks / 2) * 32, desc_lo_add(domn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0, leader);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dK += dS^T Q
-          umma_ts_w(tm_dk, tm + 64 + ks * 8, desc_lo_add(qmn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0);
-        umma_commit(&q_empty[s]);
+          umma_ts_w(tm_dk, tm + 64 + ks * 8 + (ks / 2) * 32, desc_lo_add(qmn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0, leader);
+        umma_commit(&q_empty[s], leader);
       }
-      if (ok) umma_commit(acc_done);
+      if (ok) umma_commit(acc_done, leader);
     }
   } else {
     // ------------------------------ compute warpgroups ------------------------------
-    const int wg = (warp - 2) >> 2;     // 0: even steps, 1: odd steps
+    const int wg = (warp - 2) >> 2;     // query columns [wg*32, wg*32+32) of every step
     const int quarter = warp & 3;       // TMEM lane quarter of this warp
     const int r = quarter * 32 + lane;  // key row inside the tile == TMEM lane
-    const int tid = r;
     const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
     const int kv_row = kv0 + r;
-    const uint32_t tm = tmem_base + wg * 128;
-    float* my_lse = s_lse + wg * BQ2;
-    float* my_delta = s_delta + wg * BQ2;
-    const int bar_id = 1 + wg;
-    bool ok = true;
-    // LSE (log2 domain) and Delta of a step's 64 query columns are fetched one step ahead, so their
-    // global-memory latency never sits between the score MMAs and the exponentials
-    auto load_stats = [&](int it_, float& l2_, float& dl_) {
-      l2_ = 0.f;
-      dl_ = 0.f;
-      if (tid < BQ2 && it_ < n_iter) {
-        int li_, hq_, q0_;
-        decode_iter(it_, li_, hq_, q0_);
-        const int qc = q0_ + tid;
-        const size_t idx = (size_t(b) * p.Hq + hq_) * p.S + (qc < p.S ? qc : 0);
-        l2_ = qc < p.S ? -p.lse[li_][idx] * 1.4426950408889634f : -INFINITY;   // staged negated
-        dl_ = qc < p.S ? -p.delta[li_][idx] : 0.f;
-      }
-    };
-    float l2, dl;
-    load_stats(wg, l2, dl);
-    for (int it = wg; it < n_iter; it += 2) {
-      int li, hq, q0;
-      decode_iter(it, li, hq, q0);
-      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");  // previous step's readers are done
-      if (tid < BQ2) {
-        my_lse[tid] = l2;
-        my_delta[tid] = dl;
-      }
-      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-      load_stats(it + 2, l2, dl);
-      ok = mbar_wait(&st_full[wg], (it >> 1) & 1, err);
-      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-      tc_fence_after_sync();
-      const bool diag = p.causal && (q0 < kv0 + BT);
-      uint32_t pk[32], dk[32];
-      {
-        // The staged statistics are stored negated (-LSE in the log2 domain, -Delta), so that the
-        // packed forms are plain fused multiply-adds: P = exp2(S c + (-LSE)), dS = P (dP + (-Delta)).
-        // Each half of the 64 columns: issue the TMEM loads, fetch the 32 + 32 statistics while they
-        // are in flight, then do the arithmetic on register data only.
-        const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
-        const int first_visible = diag ? kv_row - q0 : 0;  // query columns below this are masked for this key row
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t st[32], dp[32];
-          tmem_ld_x32(tm + lane_sel + h * 32, st);
-          tmem_ld_x32(tm + 64 + lane_sel + h * 32, dp);
-          ulonglong2 nl[8], nd[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            nl[i] = *reinterpret_cast<const ulonglong2*>(my_lse + h * 32 + i * 4);
-            nd[i] = *reinterpret_cast<const ulonglong2*>(my_delta + h * 32 + i * 4);
-          }
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const uint64_t x0 = ffma2(pack_f2(__uint_as_float(st[4 * i]), __uint_as_float(st[4 * i + 1])), c2, nl[i].x);
-            const uint64_t x1 = ffma2(pack_f2(__uint_as_float(st[4 * i + 2]), __uint_as_float(st[4 * i + 3])), c2, nl[i].y);
-            float e0 = fast_exp2(f2_lo(x0)), e1 = fast_exp2(f2_hi(x0));
-            float e2 = fast_exp2(f2_lo(x1)), e3 = fast_exp2(f2_hi(x1));
-            if (diag) {
-              const int col = h * 32 + i * 4;
-              e0 = col + 0 < first_visible ? 0.f : e0;
-              e1 = col + 1 < first_visible ? 0.f : e1;
-              e2 = col + 2 < first_visible ? 0.f : e2;
-              e3 = col + 3 < first_visible ? 0.f : e3;
-            }
-            pk[h * 16 + 2 * i] = pack_bf16(e0, e1);
-            pk[h * 16 + 2 * i + 1] = pack_bf16(e2, e3);
-            const uint64_t d0 = fmul2(pack_f2(e0, e1),
-                                      fadd2(pack_f2(__uint_as_float(dp[4 * i]), __uint_as_float(dp[4 * i + 1])), nd[i].x));
-            const uint64_t d1 = fmul2(pack_f2(e2, e3),
-                                      fadd2(pack_f2(__uint_as_float(dp[4 * i + 2]), __uint_as_float(dp[4 * i + 3])), nd[i].y));
-            dk[h * 16 + 2 * i] = pack_bf16(f2_lo(d0), f2_hi(d0));
-            dk[h * 16 + 2 * i + 1] = pack_bf16(f2_lo(d1), f2_hi(d1));
-          }
+    const float inv_scale = 1.f / p.scale;
+    // Statistics: in each warpgroup, lane quarter 0 stages -LSE/scale and quarter 1 stages -Delta of
+    // the warpgroup's 32 query columns.  Values are fetched two steps before they are staged, so the
+    // global-memory latency never shows.
+    const int stat_kind = quarter;  // 0 lse, 1 delta, others idle
+    uint8_t* stat_row = smem + L::OFF_STAT + (stat_kind & 1) * 2048 + (wg * 32 + lane) * 16;
+    // raw values travel in registers; the sign flip and the 1/scale are applied when a value is staged,
+    // so that nothing waits on a load in the step that issues it
+    const float stat_mul = stat_kind == 0 ? -inv_scale : -1.f;
+    const float stat_pad = stat_kind == 0 ? 30000.f * p.scale : 0.f;  // a query beyond the sequence: exp2 underflows to zero
+    int f_it = 0, f_qi = 0, f_g = 0, f_li = 0;  // step whose statistics are fetched next (incremental decode)
+    auto fetch = [&]() -> float {
+      float raw = stat_pad;
+      if (stat_kind < 2 && f_it < n_iter) {
+        const int qc = (qt_first + f_qi) * BQ2 + wg * 32 + lane;
+        if (qc < p.S) {
+          const float* src = stat_kind == 0 ? p.lse[f_li] : p.delta[f_li];
+          raw = src[(size_t(b) * p.Hq + hk * G + f_g) * p.S + qc];
         }
       }
+      ++f_it;
+      if (++f_qi == per_stream) {
+        f_qi = 0;
+        if (++f_g == G) {
+          f_g = 0;
+          ++f_li;
+        }
+      }
+      return raw;
+    };
+    auto stage = [&](int set, float raw) {
+      if (stat_kind < 2) *reinterpret_cast<uint4*>(stat_row + set * 4096) = split3_bf16(raw * stat_mul);
+    };
+    stage(0, fetch());
+    stage(1, fetch());
+    fence_proxy_async_smem();
+    mbar_arrive(stat0);
+    float s0 = fetch(), s1 = fetch();
+    const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
+    // P^T and dS^T (bf16 pairs) overwrite the first half of the warpgroup's OWN score columns: 32-bit
+    // columns [wg*48, wg*48+16) of S^T resp. dP^T, which the other warpgroup never reads
+    const uint32_t col_ld = wg * 32, col_st = wg * 48;
+    int qi = 0;  // query tile index of the current step inside its stream
+    bool ok = true;
+    for (int it = 0; it < n_iter; ++it) {
+      const int set = it & 1;
+      const uint32_t tm = tmem_base + set * 128;
+      ok = mbar_wait(&st_full[set], (it >> 1) & 1, err);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      tc_fence_after_sync();
+      uint32_t st[32], dp[32];
+      tmem_ld_x32(tm + lane_sel + col_ld, st);
+      tmem_ld_x32(tm + 64 + lane_sel + col_ld, dp);
+      // the score MMAs of this step have completed, so the set's statistics tile may take step it+2's
+      stage(set, s0);
+      s0 = s1;
+      s1 = fetch();
+      const bool diag = p.causal && qi < BT / BQ2;                  // the first two query tiles straddle the diagonal
+      const int first_visible = diag ? r - qi * BQ2 - wg * 32 : 0;  // own columns below this are masked for this key row
+      uint32_t pk[16], dk[16];
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const uint64_t x = fmul2(pack_f2(__uint_as_float(st[2 * i]), __uint_as_float(st[2 * i + 1])), c2);
+        float e0 = fast_exp2(f2_lo(x)), e1 = fast_exp2(f2_hi(x));
+        if (diag) {
+          e0 = 2 * i < first_visible ? 0.f : e0;
+          e1 = 2 * i + 1 < first_visible ? 0.f : e1;
+        }
+        pk[i] = pack_bf16(e0, e1);
+        const uint64_t d = fmul2(pack_f2(e0, e1), pack_f2(__uint_as_float(dp[2 * i]), __uint_as_float(dp[2 * i + 1])));
+        dk[i] = pack_bf16(f2_lo(d), f2_hi(d));
+      }
       // keys beyond the sequence contribute nothing (their K/V rows are zero-filled; dK/dV rows are not stored)
-      tmem_st_x32(tm + lane_sel, pk);
-      tmem_st_x32(tm + 64 + lane_sel, dk);
+      tmem_st_x16(tm + lane_sel + col_st, pk);
+      tmem_st_x16(tm + 64 + lane_sel + col_st, dk);
       tmem_st_wait();
+      fence_proxy_async_smem();  // the staged statistics are read by the tensor core's proxy
       tc_fence_before_sync();
-      mbar_arrive(&pds_ready[wg]);
+      mbar_arrive(&pds_ready[set]);
+      if (++qi == per_stream) qi = 0;
     }
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
@@ -498,7 +536,8 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
       constexpr uint32_t idesc_s = umma_idesc_bf16(BT, BT, 0, 0);
       constexpr uint32_t idesc_dq = umma_idesc_bf16(BT, DH, 0, 1);  // A = dS from TMEM, B = K MN-major
       constexpr uint32_t hi = desc_hi_sw128(1024);
@@ -511,9 +550,9 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tmem_base + x * BT, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_s, ks != 0);
+          umma_ss_w(tmem_base + x * BT, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_s, ks != 0, leader);
         }
-        umma_commit(&s_full[x]);
+        umma_commit(&s_full[x], leader);
       };
       if (ok && n_max > 0) {
         ok = mbar_wait(&k_full[0], 0, err);
@@ -536,13 +575,13 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
 #pragma unroll
             for (int ks = 0; ks < KSTEPS_DH; ++ks) {
               const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-              umma_ss_w(tmem_base + x * BT, desc_lo_add(do_lo, off), desc_lo_add(v_lo, off), hi, idesc_s, ks != 0);
+              umma_ss_w(tmem_base + x * BT, desc_lo_add(do_lo, off), desc_lo_add(v_lo, off), hi, idesc_s, ks != 0, leader);
             }
-            umma_commit(&dp_full[x]);
+            umma_commit(&dp_full[x], leader);
           }
         }
         if (!ok) break;
-        umma_commit(v_empty);
+        umma_commit(v_empty, leader);
         const bool next = j + 1 < n_max;
         if (next && !mbar_wait(&k_full[(j + 1) % DQ_KSTAGES], ((j + 1) / DQ_KSTAGES) & 1, err)) { ok = false; break; }
         const uint32_t kmn_lo = desc_lo_sw128(k_base + (j % DQ_KSTAGES) * L::TILE, HALF_BYTES);  // K_j as MN-major B
@@ -554,14 +593,14 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
 #pragma unroll
             for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ_x += dS_x(j) K_j
               umma_ts_w(tmem_base + 256 + x * 128, tmem_base + x * BT + ks * 8, desc_lo_add(kmn_lo, ks * 2048), hi,
-                        idesc_dq, (j | ks) != 0);
-            if (j + 1 == n_kv[x]) umma_commit(&dq_done[x]);
+                        idesc_dq, (j | ks) != 0, leader);
+            if (j + 1 == n_kv[x]) umma_commit(&dq_done[x], leader);
             // the tile's buffer takes the next scores right behind dQ_x(j) in the in-order tensor pipe
             if (j + 1 < n_kv[x]) issue_s(x, j + 1);
           }
         }
         if (!ok) break;
-        umma_commit(&k_empty[j % DQ_KSTAGES]);
+        umma_commit(&k_empty[j % DQ_KSTAGES], leader);
       }
     }
   } else {

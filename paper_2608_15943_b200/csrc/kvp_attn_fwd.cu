@@ -160,7 +160,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
       constexpr uint32_t idesc_qk = umma_idesc_bf16(BQ, BKV, 0, 0);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(BQ, DH, 0, 1);
       constexpr uint32_t hi = desc_hi_sw128(1024);
@@ -172,16 +173,16 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_QK; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tmem_base + x * BKV, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0);
+          umma_ss_w(tmem_base + x * BKV, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0, leader);
         }
-        umma_commit(&s_full[x]);
+        umma_commit(&s_full[x], leader);
       };
       auto issue_pv = [&](int x, int j) {  // O_x += P_x(j) V_j
         const uint32_t v_lo = desc_lo_sw128(v_base + (j % FWD_VSTAGES) * L::KV_BYTES, HALF_BYTES);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_PV; ++ks)
           umma_ts_w(tmem_base + 256 + x * 128, tmem_base + x * BKV + ks * 8, desc_lo_add(v_lo, ks * 2048), hi, idesc_pv,
-                    (j | ks) != 0);
+                    (j | ks) != 0, leader);
       };
       if (ok && n_max > 0) {
         ok = mbar_wait(&k_full[0], 0, err);
@@ -189,7 +190,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
           tc_fence_after_sync();
           if (n_kv[0] > 0) issue_s(0, 0);
           if (n_kv[1] > 0) issue_s(1, 0);
-          umma_commit(&k_empty[0]);
+          umma_commit(&k_empty[0], leader);
         }
       }
       for (int j = 0; j < n_max && ok; ++j) {
@@ -204,14 +205,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
             if (!mbar_wait(&p_ready[x], j & 1, err)) { ok = false; break; }
             tc_fence_after_sync();
             issue_pv(x, j);
-            if (j + 1 == n_kv[x]) umma_commit(&o_done[x]);
+            if (j + 1 == n_kv[x]) umma_commit(&o_done[x], leader);
             // the score buffer of tile x is free again once P_x(j) V_j has been issued (in-order pipe)
             if (j + 1 < n_kv[x]) issue_s(x, j + 1);
           }
         }
         if (!ok) break;
-        umma_commit(&v_empty[j % FWD_VSTAGES]);
-        if (next) umma_commit(&k_empty[(j + 1) % FWD_KSTAGES]);
+        umma_commit(&v_empty[j % FWD_VSTAGES], leader);
+        if (next) umma_commit(&k_empty[(j + 1) % FWD_KSTAGES], leader);
       }
     }
   } else {

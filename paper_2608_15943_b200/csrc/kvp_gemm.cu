@@ -127,7 +127,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
       uint32_t it = 0;
       uint32_t tile_i = 0;
       bool ok = true;
@@ -152,11 +153,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = smem_desc_sw128(sa + k * a_step, a_lbo, 1024);
             const uint64_t db = smem_desc_sw128(sb + k * b_step, b_lbo, 1024);
-            umma_ss(d_tmem, da, db, p.idesc, (kb | k) != 0);
+            umma_ss(d_tmem, da, db, p.idesc, (kb | k) != 0, leader);
           }
-          umma_commit(&empty[s]);  // frees the smem stage once these MMAs have read it
+          umma_commit(&empty[s], leader);  // frees the smem stage once these MMAs have read it
         }
-        if (ok) umma_commit(&acc_full[acc]);
+        if (ok) umma_commit(&acc_full[acc], leader);
       }
     }
   } else {

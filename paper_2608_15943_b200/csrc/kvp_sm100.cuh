@@ -170,31 +170,48 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, int a_mn, i
          (static_cast<uint32_t>(M >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]; one thread issues.
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
+// MMA issue.  The WHOLE (converged) warp runs the issuing code, so that addresses and descriptor
+// words stay warp-uniform values, and one elected lane executes each instruction: every issuing
+// wrapper takes that lane's predicate `leader` (nonzero in exactly one lane).  Issuing from inside
+// a divergent single-lane branch instead costs tens of cycles per instruction.
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t pred;
   asm volatile(
       "{\n"
-      " .reg .pred p;\n"
+      " .reg .pred P;\n"
+      " elect.sync _|P, 0xffffffff;\n"
+      " selp.u32 %0, 1, 0, P;\n"
+      "}\n"
+      : "=r"(pred));
+  return pred;
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate, uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p, q;\n"
       " setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      " setp.ne.b32 q, %5, 0;\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
       "}\n" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
       : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
+                                        uint32_t accumulate, uint32_t leader) {
   asm volatile(
       "{\n"
-      " .reg .pred p;\n"
+      " .reg .pred p, q;\n"
       " setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      " setp.ne.b32 q, %5, 0;\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
       "}\n" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
       : "memory");
 }
-// The same descriptor split into its two 32-bit words, so that the single MMA-issuing thread only
+// The same descriptor split into its two 32-bit words, so that the MMA-issuing warp only
 // adds a constant to the low word per instruction (the tile base and the LBO live in the low word,
 // SBO / version / swizzle mode in the high word, which is loop-invariant).
 __device__ __forceinline__ uint32_t desc_lo_sw128(uint32_t saddr, uint32_t lbo_bytes) {
@@ -207,37 +224,44 @@ __host__ __device__ constexpr uint32_t desc_hi_sw128(uint32_t sbo_bytes) {
 __device__ __forceinline__ uint32_t desc_lo_add(uint32_t lo, uint32_t byte_off) { return lo + (byte_off >> 4); }
 
 __device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
-                                          uint32_t accumulate) {
+                                          uint32_t accumulate, uint32_t leader) {
   asm volatile(
       "{\n"
-      " .reg .pred p;\n"
+      " .reg .pred p, q;\n"
       " .reg .b64 da, db;\n"
       " mov.b64 da, {%1, %3};\n"
       " mov.b64 db, {%2, %3};\n"
       " setp.ne.b32 p, %5, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
+      " setp.ne.b32 q, %6, 0;\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
       "}\n" ::"r"(d_tmem),
-      "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+      "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "r"(leader)
       : "memory");
 }
 __device__ __forceinline__ void umma_ts_w(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
-                                          uint32_t accumulate) {
+                                          uint32_t accumulate, uint32_t leader) {
   asm volatile(
       "{\n"
-      " .reg .pred p;\n"
+      " .reg .pred p, q;\n"
       " .reg .b64 db;\n"
       " mov.b64 db, {%2, %3};\n"
       " setp.ne.b32 p, %5, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n"
+      " setp.ne.b32 q, %6, 0;\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n"
       "}\n" ::"r"(d_tmem),
-      "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+      "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "r"(leader)
       : "memory");
 }
-
-// mbarrier arrives once all MMAs issued so far by this thread have completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
+// mbarrier arrives once all MMAs issued so far by the elected lane have completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar, uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred q;\n"
+      " setp.ne.b32 q, %1, 0;\n"
+      " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+      "}\n" ::"r"(smem_u32(bar)),
+      "r"(leader)
+      : "memory");
 }
 
 // ----------------------------------------------------------------------------------------

@@ -60,8 +60,8 @@ struct DkdvSmem {
   static constexpr int OFF_V = OFF_K + KV_TILE;
   static constexpr int OFF_RING = OFF_V + KV_TILE;
   static constexpr int OFF_ONES = OFF_RING + DKDV_STAGES * STAGE;  // [128 x 16] bf16, unswizzled K-major
-  static constexpr int OFF_STAT = OFF_ONES + 4096;                 // [2 sets][lse, delta][64 x 16] bf16
-  static constexpr int OFF_BAR = OFF_STAT + 4 * 2048;
+  static constexpr int OFF_STAT = OFF_ONES + 4096;                 // [4 steps][lse, delta][64 x 16] bf16
+  static constexpr int OFF_BAR = OFF_STAT + 8 * 2048;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
 
@@ -128,9 +128,11 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
   const int lane = threadIdx.x & 31;
   int* err = &g_bwd_status;
 
-  const int jt = blockIdx.x;  // key tile; tile 0 sees every query tile under the causal mask -> heaviest first
-  const int hk = blockIdx.y;
-  const int b = blockIdx.z;
+  // blocks are dispatched x-fastest: the key tile is the slowest index, so that under the causal mask the
+  // heaviest tiles (tile 0 sees every query tile) of ALL (batch, KV head) pairs start first
+  const int jt = blockIdx.z;
+  const int hk = blockIdx.x;
+  const int b = blockIdx.y;
   const int G = p.Hq / p.Hkv;
   const int kv0 = jt * BT;
   const int n_qt = (p.S + BQ2 - 1) / BQ2;
@@ -153,7 +155,7 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     mbar_fence_init();
   }
   // constant operand tiles: ones in the first three columns; statistics tiles start as zeros
-  for (int i = threadIdx.x; i < (4096 + 4 * 2048) / 16; i += blockDim.x) {
+  for (int i = threadIdx.x; i < (4096 + 8 * 2048) / 16; i += blockDim.x) {
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (i < 128) v = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);  // row i, columns 0-7 = 1,1,1,0,0,0,0,0
     *reinterpret_cast<uint4*>(smem + L::OFF_ONES + i * 16) = v;
@@ -228,7 +230,7 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         const uint32_t q_lo = desc_lo_sw128(ring + s * L::STAGE, 0);
         const uint32_t do_lo = desc_lo_sw128(ring + s * L::STAGE + L::Q_TILE, 0);
         const uint32_t tm = tmem_base + (it & 1) * 128;
-        const uint32_t stat_lo = desc_lo_plain(stat_base + (it & 1) * 4096, 1024);
+        const uint32_t stat_lo = desc_lo_plain(stat_base + (it & 3) * 4096, 1024);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
@@ -279,40 +281,66 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     // Statistics: in each warpgroup, lane quarter 0 stages -LSE/scale and quarter 1 stages -Delta of
     // the warpgroup's 32 query columns.  Values are fetched two steps before they are staged, so the
     // global-memory latency never shows.
-    const int stat_kind = quarter;  // 0 lse, 1 delta, others idle
+    const int stat_kind = quarter ^ 2;  // 0 lse, 1 delta, others idle: the warps whose scheduler hosts no TMA / MMA warp
     uint8_t* stat_row = smem + L::OFF_STAT + (stat_kind & 1) * 2048 + (wg * 32 + lane) * 16;
-    // raw values travel in registers; the sign flip and the 1/scale are applied when a value is staged,
-    // so that nothing waits on a load in the step that issues it
+    // Loads are unconditional (from a clamped, always valid address) and their raw values travel in
+    // registers together with a validity flag; sign, 1/scale and the padding value are applied when a
+    // value is staged two steps later, so that no instruction depends on a load in the step that issues it.
     const float stat_mul = stat_kind == 0 ? -inv_scale : -1.f;
-    const float stat_pad = stat_kind == 0 ? 30000.f * p.scale : 0.f;  // a query beyond the sequence: exp2 underflows to zero
-    int f_it = 0, f_qi = 0, f_g = 0, f_li = 0;  // step whose statistics are fetched next (incremental decode)
-    auto fetch = [&]() -> float {
-      float raw = stat_pad;
-      if (stat_kind < 2 && f_it < n_iter) {
-        const int qc = (qt_first + f_qi) * BQ2 + wg * 32 + lane;
-        if (qc < p.S) {
-          const float* src = stat_kind == 0 ? p.lse[f_li] : p.delta[f_li];
-          raw = src[(size_t(b) * p.Hq + hk * G + f_g) * p.S + qc];
+    const float stat_pad = stat_kind == 0 ? -30000.f : 0.f;  // a query beyond the sequence: exp2 underflows to zero
+    // Two cursors walk the steps in order (incremental decode of step -> layer, head, query tile): one
+    // for the step whose statistics are loaded next, one kStatAhead steps further that only pulls the
+    // line into L2 -- the loads are a few steps ahead of their use, which hides an L2 hit but not DRAM.
+    constexpr int kStatAhead = 12;
+    struct Cursor {
+      int it = 0, qi = 0, g = 0, li = 0;
+    };
+    auto advance = [&](Cursor& c) {
+      ++c.it;
+      if (++c.qi == per_stream) {
+        c.qi = 0;
+        if (++c.g == G) {
+          c.g = 0;
+          ++c.li;
         }
       }
-      ++f_it;
-      if (++f_qi == per_stream) {
-        f_qi = 0;
-        if (++f_g == G) {
-          f_g = 0;
-          ++f_li;
-        }
+    };
+    const float* f_ptr = p.lse[0];
+    auto locate = [&](const Cursor& c, bool& valid) {  // address of this lane's statistic of step c (clamped, always valid)
+      valid = false;
+      if (stat_kind < 2 && c.it < n_iter) {
+        const int qc = (qt_first + c.qi) * BQ2 + wg * 32 + lane;
+        valid = qc < p.S;
+        const float* src = stat_kind == 0 ? p.lse[c.li] : p.delta[c.li];
+        f_ptr = src + (size_t(b) * p.Hq + hk * G + c.g) * p.S + (valid ? qc : p.S - 1);
       }
-      return raw;
+      return f_ptr;
     };
-    auto stage = [&](int set, float raw) {
-      if (stat_kind < 2) *reinterpret_cast<uint4*>(stat_row + set * 4096) = split3_bf16(raw * stat_mul);
+    Cursor cf, cp;
+    for (int i = 0; i < kStatAhead; ++i) advance(cp);
+    auto fetch = [&](bool& valid) -> float {
+      bool ahead_valid;
+      const float* ahead = locate(cp, ahead_valid);
+      if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(ahead));
+      advance(cp);
+      const float* ptr = locate(cf, valid);
+      advance(cf);
+      return __ldg(ptr);
     };
-    stage(0, fetch());
-    stage(1, fetch());
+    auto stage = [&](int tile, float raw, bool valid) {
+      if (stat_kind < 2) *reinterpret_cast<uint4*>(stat_row + tile * 4096) = split3_bf16(valid ? raw * stat_mul : stat_pad);
+    };
+    bool v0, v1;
+    float s0, s1;
+#pragma unroll 1
+    for (int i = 0; i < 3; ++i) {  // the tiles of steps 0..2; step n+3's tile is staged at the end of step n
+      s0 = fetch(v0);
+      stage(i, s0, v0);
+    }
     fence_proxy_async_smem();
     mbar_arrive(stat0);
-    float s0 = fetch(), s1 = fetch();
+    s0 = fetch(v0);
+    s1 = fetch(v1);
     const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
     // P^T and dS^T (bf16 pairs) overwrite the first half of the warpgroup's OWN score columns: 32-bit
     // columns [wg*48, wg*48+16) of S^T resp. dP^T, which the other warpgroup never reads
@@ -328,10 +356,9 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
       uint32_t st[32], dp[32];
       tmem_ld_x32(tm + lane_sel + col_ld, st);
       tmem_ld_x32(tm + 64 + lane_sel + col_ld, dp);
-      // the score MMAs of this step have completed, so the set's statistics tile may take step it+2's
-      stage(set, s0);
-      s0 = s1;
-      s1 = fetch();
+      // issued here, so that the load has returned before the fences below (which wait for it)
+      bool v_new;
+      const float s_new = fetch(v_new);
       const bool diag = p.causal && qi < BT / BQ2;                  // the first two query tiles straddle the diagonal
       const int first_visible = diag ? r - qi * BQ2 - wg * 32 : 0;  // own columns below this are masked for this key row
       uint32_t pk[16], dk[16];
@@ -352,9 +379,16 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
       tmem_st_x16(tm + lane_sel + col_st, pk);
       tmem_st_x16(tm + 64 + lane_sel + col_st, dk);
       tmem_st_wait();
-      fence_proxy_async_smem();  // the staged statistics are read by the tensor core's proxy
+      fence_proxy_async_smem();  // the statistics staged one step ago are read by the tensor core's proxy
       tc_fence_before_sync();
       mbar_arrive(&pds_ready[set]);
+      // Off the critical path: the tile of step it+3 (last read by the scores of step it-1, which have
+      // completed).  The next step's arrive publishes it, before the scores of step it+3 are issued.
+      stage((it + 3) & 3, s0, v0);
+      s0 = s1;
+      v0 = v1;
+      s1 = s_new;
+      v1 = v_new;
       if (++qi == per_stream) qi = 0;
     }
     ok = __all_sync(0xffffffffu, ok);
@@ -878,7 +912,7 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     p.causal = causal;
     p.scale = sc;
     p.scale_log2 = sc * 1.4426950408889634f;
-    dim3 grid((s->S + BT - 1) / BT, s->Hkv, s->B);
+    dim3 grid(s->Hkv, s->B, (s->S + BT - 1) / BT);
     timing_before(KVP_KERNEL_ATTN_BWD, stream);
     if (dh == 128)
       dkdv_kernel<128><<<grid, DKDV_THREADS, DkdvSmem<128>::TOTAL, stream>>>(p);

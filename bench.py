@@ -147,7 +147,7 @@ class TrainRunner:
         if out_proj and backward:
             self.d_o = [torch.empty_like(x) for x in self.out["o"]]
 
-    def step(self, _i=0):
+    def step(self, _i=0, before_proj_bwd=None):
         k, c, t, o = self.kvp, self.cfg, self.t, self.out
         k.proj_fwd(self.sh, c.donor, t["x"], t["wq"], t["wk"], t["wv"], o["q"], o["k"], o["v"])
         k.attn_fwd(self.sh, c.donor, o["q"], o["k"], o["v"], o["o"], o["lse"])
@@ -161,6 +161,8 @@ class TrainRunner:
             d_o = self.d_o
         k.attn_bwd(self.sh, c.donor, o["q"], o["k"], o["v"], o["o"], d_o, o["lse"], o["dq"], o["dk_sum"],
                    o["dv_sum"], self.ws)
+        if before_proj_bwd is not None:
+            before_proj_bwd()
         k.proj_bwd(self.sh, c.donor, t["x"], t["wq"], t["wk"], t["wv"], o["dq"], o["dk_sum"], o["dv_sum"],
                    o["dwq"], o["dwk"], o["dwv"], o["dx"], self.ws)
         if self.bucket is not None:
@@ -179,21 +181,63 @@ class TrainRunner:
         f = c.proj_fwd_flops() + (c.L * 2 * c.T * c.D * c.Hq * c.dh if self.out_proj else 0)
         return 3 * f if self.backward else f
 
-    # end-to-end: the step's inputs come from pinned host memory, the block's dX goes back
+    # End to end: every step's inputs come from pinned host memory and the block's dX goes back.  The copies
+    # are pipelined the way an input loader does it: while step n computes, a second stream brings step
+    # n+1's inputs into the other of two device buffer sets, and a third takes step n's result out.  Every
+    # call issues exactly one input copy and one result copy and does not return the compute stream until
+    # the input copy it issued has landed, so K timed calls contain K input and K result transfers.
     def setup_e2e(self):
         names = ["x", "dy" if self.out_proj else "d_o"] if self.backward else ["x"]
+        self.e2e_names = names
         self.h_in = {n: [a.cpu().pin_memory() for a in self.t[n]] for n in names}
+        self.in_sets = [{n: self.t[n] for n in names}, {n: [torch.empty_like(a) for a in self.t[n]] for n in names}]
         self.h_out = torch.empty_like(self.out["dx"][0] if self.backward else self.out["o"][-1],
                                       device="cpu").pin_memory()
         self.h2d = sum(a.numel() * a.element_size() for n in names for a in self.h_in[n])
         self.d2h = self.h_out.numel() * self.h_out.element_size()
+        self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        self.ev_in = [torch.cuda.Event(), torch.cuda.Event()]      # input set filled
+        self.ev_free = [torch.cuda.Event(), torch.cuda.Event()]    # input set no longer read
+        self.ev_result, self.ev_out = torch.cuda.Event(), torch.cuda.Event()
+        self.e2e_calls = 0
+        cur = torch.cuda.current_stream()
+        self._copy_in(0, after=None)           # the first call's inputs
+        cur.wait_event(self.ev_in[0])
+        self.ev_out.record(cur)
+
+    def _copy_in(self, which, after):
+        with torch.cuda.stream(self.s_in):
+            if after is not None:
+                self.s_in.wait_event(after)    # the set's previous reader has finished
+            for n in self.e2e_names:
+                for dst, src in zip(self.in_sets[which][n], self.h_in[n]):
+                    dst.copy_(src, non_blocking=True)
+            self.ev_in[which].record(self.s_in)
 
     def step_e2e(self, _i=0):
-        for n, hs in self.h_in.items():
-            for dst, src in zip(self.t[n], hs):
-                dst.copy_(src, non_blocking=True)
-        self.step()
-        self.h_out.copy_(self.out["dx"][0] if self.backward else self.out["o"][-1], non_blocking=True)
+        cur = torch.cuda.current_stream()
+        a = self.e2e_calls & 1
+        self.e2e_calls += 1
+        for n in self.e2e_names:
+            self.t[n] = self.in_sets[a][n]
+        # next step's inputs into the other set, once the step before this one has stopped reading it
+        self._copy_in(1 - a, after=self.ev_free[1 - a] if self.e2e_calls > 1 else None)
+        result = self.out["dx"][0] if self.backward else self.out["o"][-1]
+        # the previous result must have left the device before this step overwrites it
+        if self.backward:
+            self.step(before_proj_bwd=lambda: cur.wait_event(self.ev_out))
+        else:
+            cur.wait_event(self.ev_out)
+            self.step()
+        self.ev_free[a].record(cur)
+        self.ev_result.record(cur)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_result)
+            self.h_out.copy_(result, non_blocking=True)
+            self.ev_out.record(self.s_out)
+        cur.wait_event(self.ev_in[1 - a])      # the copy issued by this call is inside this call's time
+        if _i == getattr(self, "e2e_last", -1):  # the last timed call also waits for its own result copy
+            cur.wait_event(self.ev_out)
 
 
 def cpu_baseline_train(cfg: W.TrainCfg, backward: bool, heads: int = 4, proj_tokens: int = 1024):
@@ -379,6 +423,7 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
         for i in range(2):
             runner.step_e2e(i)
         e2e_steps = max(3, min(args.steps, 5))
+        runner.e2e_last = e2e_steps - 1
         ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
         e2e_val = world * flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
     status = kvp.device_status()
@@ -396,7 +441,9 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
         "pct_bf16_peak_nominal": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
         "pct_bf16_peak_measured": 100.0 * value / world / peak,
         "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": runner.h2d,
-                "d2h_bytes_per_step": runner.d2h, "ms_per_step": ms_e2e / e2e_steps},
+                "d2h_bytes_per_step": runner.d2h, "ms_per_step": ms_e2e / e2e_steps,
+                "copies": "pipelined: step n+1's inputs arrive on a second stream while step n computes; "
+                          "one input and one result transfer per timed step"},
         "roofline": roofline, "device_status": kvp.status_string(status),
     }
     del runner

@@ -227,7 +227,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
     const int my_n = n_kv[x];
     const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
     float m_used = -INFINITY;  // running maximum (log2 domain) the exponentials are taken against
-    uint64_t l2 = 0ull;        // two partial row sums (packed lanes)
+    uint64_t l2 = 0ull, l2b = 0ull;  // four partial row sums (two packed pairs, for independent add chains)
     bool ok = true;
     for (int j = 0; j < my_n; ++j) {
       ok = mbar_wait(&s_full[x], j & 1, err);
@@ -248,9 +248,15 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         for (int i = 0; i < BKV; ++i)
           if (i >= lim) sv[i] = 0xff800000u;  // -inf
       }
-      float m_raw = fmaxf(__uint_as_float(sv[0]), __uint_as_float(sv[1]));
+      // four independent partial maxima: one 64-deep dependent chain would cost its full latency per tile
+      float mp[4];
 #pragma unroll
-      for (int i = 2; i < BKV; i += 2) m_raw = fmax3(m_raw, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+      for (int u = 0; u < 4; ++u) mp[u] = fmaxf(__uint_as_float(sv[2 * u]), __uint_as_float(sv[2 * u + 1]));
+#pragma unroll
+      for (int i = 8; i < BKV; i += 8)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mp[u] = fmax3(mp[u], __uint_as_float(sv[i + 2 * u]), __uint_as_float(sv[i + 2 * u + 1]));
+      const float m_raw = fmaxf(fmaxf(mp[0], mp[1]), fmaxf(mp[2], mp[3]));
       const float m_tile = m_raw * p.scale_log2;  // the scale is positive, so the maximum commutes with it
       float alpha = 1.f;
       bool rescale = false;
@@ -260,6 +266,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         alpha = fast_exp2(m_used - m_tile);
         m_used = m_tile;
         l2 = fmul2(l2, pack_f2(alpha, alpha));
+        l2b = fmul2(l2b, pack_f2(alpha, alpha));
         rescale = true;
       }
       const uint64_t nm2 = pack_f2(-m_used, -m_used);
@@ -269,9 +276,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
           const uint64_t t = ffma2(pack_f2(__uint_as_float(sv[c * 32 + 2 * i]), __uint_as_float(sv[c * 32 + 2 * i + 1])), c2, nm2);
-          const float e0 = fast_exp2(f2_lo(t)), e1 = fast_exp2(f2_hi(t));
-          l2 = fadd2(l2, pack_f2(e0, e1));
-          pk[i] = pack_bf16(e0, e1);
+          const uint64_t e = pack_f2(fast_exp2(f2_lo(t)), fast_exp2(f2_hi(t)));
+          if (i & 1) l2b = fadd2(l2b, e); else l2 = fadd2(l2, e);
+          pk[i] = pack_bf16(f2_lo(e), f2_hi(e));
         }
         tmem_st_x16(tm_s + c * 16, pk);  // P as bf16 pairs over the first 64 columns of the score buffer
       }
@@ -298,7 +305,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
     }
     if (ok && my_n > 0) {
       tc_fence_after_sync();
-      const float l_sum = f2_lo(l2) + f2_hi(l2);
+      const float l_sum = (f2_lo(l2) + f2_hi(l2)) + (f2_lo(l2b) + f2_hi(l2b));
       const float inv_l = 1.f / l_sum;
       const bool valid = q_row < p.S;
       __nv_bfloat16* dst = p.o + ((size_t(b) * p.S + (valid ? q_row : 0)) * p.Hq + hq) * DH;

@@ -122,6 +122,27 @@ typedef struct {
 } kvp_model_desc;
 int kvp_layer_flops(const kvp_model_desc* m, uint64_t* f_full, uint64_t* f_share, uint64_t* f_lm_head);
 
+/* 1F1B pipeline timing model (host only, pure, exact integer arithmetic).
+ *
+ * The paper measures KV-Pipe under the non-interleaved 1F1B schedule (section "Results on Ascend
+ * 910B NPUs") and ties the iteration time to the stage imbalance FIR (Eq. 4-5); it prints no timing
+ * model.  kvp_sim_1f1b evaluates that schedule for given per-stage times: stage i of P runs
+ * min(P-1-i, M) warm-up forwards, then alternates one forward and one backward, then drains its
+ * remaining backwards, strictly in that order; forward (i, m) needs forward (i-1, m), backward (i, m)
+ * needs backward (i+1, m) (its own forward on the last stage); transfers cost nothing.  An operation
+ * starts when its inputs exist and the stage is free.
+ *
+ * t_fwd / t_bwd: host [P], time of one micro-batch on stage i, any unit, >= 0.  out->makespan is the
+ * finish time of the last operation; out->idle (host [P], may be NULL) receives
+ * makespan - M * (t_fwd[i] + t_bwd[i]), the stage's bubble.  P >= 1, M >= 1 and P * M <= 2^24, else
+ * KVP_ERR_INVALID_ARG.  Feeding measured stage times of a converted and an unconverted stage gives the
+ * iteration-time effect of a plan without a multi-device run. */
+typedef struct {
+  int64_t makespan;
+  int64_t* idle;
+} kvp_sim_out;
+int kvp_sim_1f1b(int32_t P, int32_t M, const int64_t* t_fwd, const int64_t* t_bwd, kvp_sim_out* out);
+
 /* ------------------------------------------------------------------------------------------
  * Training / prefill path
  * ---------------------------------------------------------------------------------------- */

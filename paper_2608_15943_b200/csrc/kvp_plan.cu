@@ -2,6 +2,7 @@
 // (architecture-balanced, tail-first, bottleneck-retargeting conversion), the safe-layer
 // guardrail, the two comparison placements, the donor map and the analytic FLOPs helper.
 // Pure host code in exact integer arithmetic (128-bit products), off the hot path.
+#include <algorithm>
 #include <vector>
 
 #include "kvp_host.h"
@@ -213,5 +214,59 @@ extern "C" int kvp_plan(const kvp_plan_in* in, kvp_plan_out* out) {
   out->fir = double(f.num) / double(f.den);
   out->n_conv = t;
   out->stop_reason = reason;
+  return KVP_OK;
+}
+
+// 1F1B timing model.  Event-driven: every stage keeps a cursor into its operation sequence and a clock; a
+// sweep over the stages executes every operation whose remote input has been produced, until nothing is
+// left.  Finish times of forwards and backwards live in two P x M tables (-1 = not produced yet).
+extern "C" int kvp_sim_1f1b(int32_t P, int32_t M, const int64_t* t_fwd, const int64_t* t_bwd, kvp_sim_out* out) {
+  if (P < 1 || M < 1 || t_fwd == nullptr || t_bwd == nullptr || out == nullptr) return KVP_ERR_INVALID_ARG;
+  if (int64_t(P) * int64_t(M) > (int64_t(1) << 24)) return KVP_ERR_INVALID_ARG;
+  for (int i = 0; i < P; ++i)
+    if (t_fwd[i] < 0 || t_bwd[i] < 0) return KVP_ERR_INVALID_ARG;
+  std::vector<int64_t> fin_f(size_t(P) * M, -1), fin_b(size_t(P) * M, -1), clock(P, 0);
+  std::vector<int32_t> next_f(P, 0), next_b(P, 0);  // micro-batch of the stage's next forward / backward
+  int64_t remaining = int64_t(2) * P * M;
+  while (remaining > 0) {
+    bool progressed = false;
+    for (int i = 0; i < P; ++i) {
+      for (;;) {
+        if (next_f[i] >= M && next_b[i] >= M) break;
+        const int warm = std::min(P - 1 - i, M);
+        // position in the sequence: warm-up forwards, then (F, B) pairs, then the draining backwards
+        bool forward;
+        if (next_f[i] < warm) forward = true;
+        else if (next_f[i] < M) forward = (next_f[i] - warm == next_b[i]);  // pair k = F(warm+k) then B(k)
+        else forward = false;
+        if (forward) {
+          const int m = next_f[i];
+          int64_t ready = 0;
+          if (i > 0) {
+            ready = fin_f[size_t(i - 1) * M + m];
+            if (ready < 0) break;
+          }
+          clock[i] = std::max(clock[i], ready) + t_fwd[i];
+          fin_f[size_t(i) * M + m] = clock[i];
+          ++next_f[i];
+        } else {
+          const int m = next_b[i];
+          const int64_t ready = i + 1 < P ? fin_b[size_t(i + 1) * M + m] : fin_f[size_t(i) * M + m];
+          if (ready < 0) break;
+          clock[i] = std::max(clock[i], ready) + t_bwd[i];
+          fin_b[size_t(i) * M + m] = clock[i];
+          ++next_b[i];
+        }
+        --remaining;
+        progressed = true;
+      }
+    }
+    if (!progressed) return KVP_ERR_UNSUPPORTED;  // cannot happen for this schedule; never spin
+  }
+  int64_t makespan = 0;
+  for (int i = 0; i < P; ++i) makespan = std::max(makespan, clock[i]);
+  out->makespan = makespan;
+  if (out->idle != nullptr)
+    for (int i = 0; i < P; ++i) out->idle[i] = makespan - int64_t(M) * (t_fwd[i] + t_bwd[i]);
   return KVP_OK;
 }

@@ -25,7 +25,7 @@ PLACE_ARCH_BALANCED, PLACE_UNIFORM, PLACE_BIPOLAR = range(3)
 OP_PROJ_FWD, OP_PROJ_BWD, OP_ATTN_FWD, OP_ATTN_BWD, OP_DECODE = range(5)
 
 EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events",
-           "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_workspace_bytes",
+           "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_sim_1f1b", "kvp_workspace_bytes",
            "kvp_proj_fwd", "kvp_proj_bwd", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
            "kvp_gemm", "kvp_decode_workspace_bytes", "kvp_cache_append", "kvp_decode", "kvp_decode_static"]
 
@@ -153,6 +153,25 @@ def layer_flops(h, f, a, g, dh, s, vocab, causal_half=True):
     o = [C.c_uint64() for _ in range(3)]
     _check(lib.kvp_layer_flops(C.byref(m), *[C.byref(x) for x in o]), "kvp_layer_flops")
     return tuple(int(x.value) for x in o)
+
+
+class _SimOut(C.Structure):
+    _fields_ = [("makespan", C.c_int64), ("idle", C.POINTER(C.c_int64))]
+
+
+lib.kvp_sim_1f1b.restype = C.c_int
+lib.kvp_sim_1f1b.argtypes = [C.c_int32, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(_SimOut)]
+
+
+def sim_1f1b(t_fwd, t_bwd, M):
+    """kvp_sim_1f1b -> (makespan, idle[P]) for per-stage forward / backward times (integers) and M micro-batches."""
+    P = len(t_fwd)
+    tf = (C.c_int64 * P)(*[int(x) for x in t_fwd])
+    tb = (C.c_int64 * len(t_bwd))(*[int(x) for x in t_bwd])
+    idle = (C.c_int64 * max(P, 1))()
+    out = _SimOut(0, idle)
+    _check(lib.kvp_sim_1f1b(P if len(t_bwd) == P else -1, int(M), tf, tb, C.byref(out)), "kvp_sim_1f1b")
+    return int(out.makespan), [int(x) for x in idle[:P]]
 
 
 # ------------------------------------------------------------------------------------------

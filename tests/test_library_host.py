@@ -135,3 +135,25 @@ def test_plan_rejects_bad_input(kvp):
         kvp.plan([0, 2, 4], [10] * 4, [5] * 4, [0, 0], eps=(1, 0))  # zero denominator
     with pytest.raises(kvp.KvpError):
         kvp.plan([0, 2, 4], [2 ** 63] * 4, [5] * 4, [0, 0])        # totals overflow 64 bits
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_sim_1f1b_bit_exact_against_oracle(kvp, seed):
+    import random
+    from oracle import pipeline as PL
+    rng = random.Random(seed)
+    for _ in range(40):
+        P, M = rng.randint(1, 9), rng.randint(1, 12)
+        tf = [rng.randint(0, 10 ** 6) for _ in range(P)]
+        tb = [rng.randint(0, 2 * 10 ** 6) for _ in range(P)]
+        assert kvp.sim_1f1b(tf, tb, M) == tuple(PL.sim_1f1b(tf, tb, M))
+    # the paper's setting: 8 stages, the last one heavier
+    tf, tb = [100] * 7 + [118], [200] * 7 + [236]
+    assert kvp.sim_1f1b(tf, tb, 32) == tuple(PL.sim_1f1b(tf, tb, 32))
+    assert kvp.sim_1f1b([5] * 8, [10] * 8, 16)[0] == (16 + 7) * 15
+
+
+def test_sim_1f1b_rejects_bad_input(kvp):
+    for args in (([], [], 4), ([1, 2], [1], 4), ([1, 2], [1, 2], 0), ([1, -2], [1, 2], 3)):
+        with pytest.raises(kvp.KvpError):
+            kvp.sim_1f1b(*args)

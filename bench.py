@@ -515,6 +515,47 @@ def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, st
     return out
 
 
+def run_decode_sweep(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
+    """The paper's inference case study as a workload shape: LLaMA2-7B geometry with MHA (32 KV heads, so a
+    converted layer saves four times the bytes of the GQA case), context 8K ... 128K, half of the layers
+    sharing the K/V of the layer below, against the same model with every layer storing its own K/V."""
+    B, steps, warmup = 4, 16, 3
+    rows = []
+    for ctx in (8192, 16384, 32768, 65536, 131072):
+        row = {"context": ctx}
+        for key, donor in (("shared_50pct", W.pair_donor(32, 0)), ("unshared", list(range(32)))):
+            cfg = W.DecodeCfg(f"sweep-mha-{key}-{ctx}", 32, B, 32, 32, 128, 128, ctx, ctx, donor, steps)
+            own = len(cfg.owners())
+            free, _total = torch.cuda.mem_get_info()
+            pages = B * ((ctx + steps + cfg.page - 1) // cfg.page)
+            per_slot = 2 * pages * cfg.Hkv * cfg.page * cfg.dh * 2
+            n_slots = int(max(1, min(own, (free - (6 << 30)) // per_slot)))
+            runner = DecodeRunner(kvp, cfg, device, n_slots=n_slots)
+            for i in range(warmup):
+                runner.step(i)
+            torch.cuda.synchronize()
+            runner.reset()
+            with kvp.KernelTimer(kvp.KERNEL_DECODE, steps) as kt:
+                ms, clocks = timed_region(runner.step, steps, device, local_rank)
+            k_ms = float(np.mean(kt.durations_ms()))
+            step_bytes = W.decode_step_bytes(cfg, [ctx + (steps + 1) / 2.0] * B)
+            row[key] = {"tokens_per_s": world * B / (ms / steps * 1e-3), "ms_per_step": ms / steps, "stored_layers": own,
+                        "physical_layer_pools": n_slots, "bytes_per_step": step_bytes,
+                        "kernel_gbs": step_bytes / (k_ms * 1e-3) / 1e9, "frac_of_measured_copy": step_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                        "sm_mhz": clocks.get("sm_mhz")}
+            del runner
+            torch.cuda.empty_cache()
+        row["speedup_shared"] = row["shared_50pct"]["tokens_per_s"] / row["unshared"]["tokens_per_s"]
+        rows.append(row)
+    last = rows[-1]["shared_50pct"]
+    return {"metric": "shared-cache decode tokens/s (MHA, 128K context, 50% sharing)", "value": last["tokens_per_s"],
+            "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": last["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "decode-sweep-LLaMA2-7B-MHA", "layers": 32, "heads": [32, 32], "head_dim": 128,
+                       "batch_per_gpu": B, "page": 128, "l2": "cache slices far larger than L2"},
+            "sweep": rows, "device_status": kvp.status_string(kvp.device_status())}
+
+
 def run_stage(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
     """Tail pipeline stage of the planned 32-layer decoder: full attention block (Q/K/V projections,
     attention, output projection) forward + backward, converted (stage-local donor) vs unconverted."""
@@ -666,7 +707,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="train", choices=["train", "prefill", "decode", "stage", "pipeline"])
+    ap.add_argument("--workload", default="train", choices=["train", "prefill", "decode", "stage", "pipeline", "decode_sweep"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode workload in the default run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -701,6 +742,8 @@ def main():
             line["cpu_baseline"] = cpu_baseline_train(cfg, backward)
             if "decode" in line and "error" not in line["decode"]:
                 line["decode"]["cpu_baseline"] = cpu_baseline_decode(W.C3)
+    elif args.workload == "decode_sweep":
+        line = run_decode_sweep(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
     elif args.workload == "pipeline":
         line = run_pipeline(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
     elif args.workload == "decode":

@@ -76,6 +76,7 @@ struct DkdvParams {
   int n_layers;
   int B, S, Hq, Hkv;
   int causal;
+  int chunk;                      // (batch, KV head) pairs per dispatch chunk
   float scale;
   float scale_log2;
 };
@@ -128,11 +129,19 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
   const int lane = threadIdx.x & 31;
   int* err = &g_bwd_status;
 
-  // blocks are dispatched x-fastest: the key tile is the slowest index, so that under the causal mask the
-  // heaviest tiles (tile 0 sees every query tile) of ALL (batch, KV head) pairs start first
-  const int jt = blockIdx.z;
-  const int hk = blockIdx.x;
-  const int b = blockIdx.y;
+  // Blocks are dispatched in index order.  The (batch, KV head) pairs are taken in chunks of p.chunk pairs;
+  // inside a chunk the key tile is the slow index, so that under the causal mask the chunk's heaviest tiles
+  // (tile 0 sees every query tile) start first, while all CTAs that stream the same Q / dO tiles run within
+  // a wave or two of each other and find them in L2.
+  const int n_jt = (p.S + BT - 1) / BT;
+  const int n_pairs = p.Hkv * p.B;
+  const int chunk_i = blockIdx.x / (p.chunk * n_jt);
+  const int in_chunk = blockIdx.x - chunk_i * p.chunk * n_jt;
+  const int chunk_n = min(p.chunk, n_pairs - chunk_i * p.chunk);  // the last chunk may be short
+  const int jt = in_chunk / chunk_n;
+  const int pair = chunk_i * p.chunk + (in_chunk - jt * chunk_n);
+  const int hk = pair % p.Hkv;
+  const int b = pair / p.Hkv;
   const int G = p.Hq / p.Hkv;
   const int kv0 = jt * BT;
   const int n_qt = (p.S + BQ2 - 1) / BQ2;
@@ -912,7 +921,15 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     p.causal = causal;
     p.scale = sc;
     p.scale_log2 = sc * 1.4426950408889634f;
-    dim3 grid(s->Hkv, s->B, (s->S + BT - 1) / BT);
+    // chunk: the smallest divisor of the pair count that still fills the SMs 1.5 times with CTAs
+    const int n_jt = (s->S + BT - 1) / BT, n_pairs = s->Hkv * s->B;
+    p.chunk = n_pairs;
+    for (int d = 1; d <= n_pairs; ++d)
+      if (n_pairs % d == 0 && 2 * d * n_jt >= 3 * sm_count()) {
+        p.chunk = d;
+        break;
+      }
+    dim3 grid(n_pairs * n_jt);
     timing_before(KVP_KERNEL_ATTN_BWD, stream);
     if (dh == 128)
       dkdv_kernel<128><<<grid, DKDV_THREADS, DkdvSmem<128>::TOTAL, stream>>>(p);

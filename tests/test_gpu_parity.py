@@ -168,6 +168,10 @@ SHAPES = [
     (1, 384, 8, 2, 128, [0, 0, 0], True),
     (2, 300, 4, 4, 128, [0, 1, 1], False),
     (1, 515, 4, 1, 64, [0, 0], True),
+    (1, 64, 2, 2, 128, [0], True),                          # exactly one 64-query step, MHA
+    (1, 65, 2, 1, 128, [0, 0], False),
+    (3, 200, 6, 3, 128, [0, 0, 0, 0, 0, 0, 0, 0], True),    # the largest donor group (8 layers), odd pair count
+    (2, 193, 4, 4, 64, [0, 1, 1, 3], False),                # MHA (G = 1), mixed groups
 ]
 
 

@@ -204,6 +204,25 @@ int kvp_gemm(int M, int N, int K, const void* a, int64_t lda, int a_mn, const vo
              void* c, int64_t ldc, int out_f32, kvp_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Element-wise operators of a decoder stage.
+ *
+ * The paper's stage tables list a forward time per pipeline stage of LLaMA2-7B but define no operator
+ * besides attention (Eq. 1-3); these are the published definitions of the architecture it names, provided
+ * so that a whole stage's forward pass can be timed with this library.  Device pointers, 16-byte aligned,
+ * bf16 storage, fp32 arithmetic, asynchronous on `stream`; `out` may alias an input.
+ *   kvp_rmsnorm  y[T,D] = x / sqrt(mean_D(x^2) + eps) * w[D]; D a multiple of 8, D <= 8192.
+ *   kvp_rope     in place on x [B,S,H,dh]: consecutive pairs (x[2i], x[2i+1]) of every head are rotated by
+ *                (pos0 + s) * theta^(-2i/dh); dh a multiple of 8, dh <= 256, pos0 + S <= 2^18.
+ *   kvp_swiglu   out[n] = silu(gate) * up, silu(t) = t / (1 + exp(-t)); n a multiple of 8.
+ *   kvp_add      out[n] = a + b; n a multiple of 8.
+ * KVP_ERR_INVALID_ARG for null pointers / negative sizes, KVP_ERR_UNSUPPORTED for the shape limits.
+ * ---------------------------------------------------------------------------------------- */
+int kvp_rmsnorm(int32_t T, int32_t D, const void* x, const void* w, float eps, void* y, kvp_stream_t stream);
+int kvp_rope(int32_t B, int32_t S, int32_t H, int32_t dh, float theta, int32_t pos0, void* x, kvp_stream_t stream);
+int kvp_swiglu(int64_t n, const void* gate, const void* up, void* out, kvp_stream_t stream);
+int kvp_add(int64_t n, const void* a, const void* b, void* out, kvp_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
  * Decode over the shared paged cache
  * ---------------------------------------------------------------------------------------- */
 typedef struct {

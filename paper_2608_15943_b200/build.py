@@ -16,7 +16,7 @@ OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libkvp.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 
-SOURCES = ["kvp_common.cu", "kvp_plan.cu", "kvp_gemm.cu", "kvp_attn_fwd.cu", "kvp_attn_bwd.cu", "kvp_decode.cu", "kvp_misc.cu",
+SOURCES = ["kvp_common.cu", "kvp_plan.cu", "kvp_gemm.cu", "kvp_attn_fwd.cu", "kvp_attn_bwd.cu", "kvp_decode.cu", "kvp_misc.cu", "kvp_stage.cu",
            "kvp_api.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "--expt-relaxed-constexpr", "-Xptxas", "-v"] + os.environ.get("KVP_NVCC_EXTRA", "").split()

@@ -27,7 +27,8 @@ OP_PROJ_FWD, OP_PROJ_BWD, OP_ATTN_FWD, OP_ATTN_BWD, OP_DECODE = range(5)
 EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events",
            "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_sim_1f1b", "kvp_workspace_bytes",
            "kvp_proj_fwd", "kvp_proj_bwd", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
-           "kvp_gemm", "kvp_decode_workspace_bytes", "kvp_cache_append", "kvp_decode", "kvp_decode_static"]
+           "kvp_gemm", "kvp_rmsnorm", "kvp_rope", "kvp_swiglu", "kvp_add", "kvp_decode_workspace_bytes", "kvp_cache_append",
+           "kvp_decode", "kvp_decode_static"]
 
 
 class KvpError(RuntimeError):
@@ -97,6 +98,45 @@ def gemm(a: torch.Tensor, b: torch.Tensor, c: torch.Tensor, a_mn: bool = False, 
     _check(lib.kvp_gemm(M, N, K, a.data_ptr(), a.stride(0), int(a_mn), b.data_ptr(), b.stride(0), int(b_mn),
                         c.data_ptr(), c.stride(0), int(c.dtype == torch.float32), _stream()), "kvp_gemm")
     return c
+
+
+# ------------------------------------------------------------------------------------------
+# element-wise stage operators
+# ------------------------------------------------------------------------------------------
+lib.kvp_rmsnorm.restype = C.c_int
+lib.kvp_rmsnorm.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p]
+lib.kvp_rope.restype = C.c_int
+lib.kvp_rope.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_int32, C.c_void_p, C.c_void_p]
+lib.kvp_swiglu.restype = C.c_int
+lib.kvp_swiglu.argtypes = [C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.kvp_add.restype = C.c_int
+lib.kvp_add.argtypes = [C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+
+
+def rmsnorm(x: torch.Tensor, w: torch.Tensor, eps: float, y: torch.Tensor) -> torch.Tensor:
+    """kvp_rmsnorm: y[T,D] = x / sqrt(mean(x^2) + eps) * w (bf16)."""
+    T, D = x.shape
+    _check(lib.kvp_rmsnorm(T, D, x.data_ptr(), w.data_ptr(), float(eps), y.data_ptr(), _stream()), "kvp_rmsnorm")
+    return y
+
+
+def rope(x: torch.Tensor, theta: float = 10000.0, pos0: int = 0) -> torch.Tensor:
+    """kvp_rope: in place on x [B,S,H,dh] (bf16)."""
+    B, S, H, dh = x.shape
+    _check(lib.kvp_rope(B, S, H, dh, float(theta), int(pos0), x.data_ptr(), _stream()), "kvp_rope")
+    return x
+
+
+def swiglu(gate: torch.Tensor, up: torch.Tensor, out: torch.Tensor) -> torch.Tensor:
+    """kvp_swiglu: out = silu(gate) * up (bf16, same shapes)."""
+    _check(lib.kvp_swiglu(gate.numel(), gate.data_ptr(), up.data_ptr(), out.data_ptr(), _stream()), "kvp_swiglu")
+    return out
+
+
+def add(a: torch.Tensor, b: torch.Tensor, out: torch.Tensor) -> torch.Tensor:
+    """kvp_add: out = a + b (bf16, same shapes)."""
+    _check(lib.kvp_add(a.numel(), a.data_ptr(), b.data_ptr(), out.data_ptr(), _stream()), "kvp_add")
+    return out
 
 
 # ------------------------------------------------------------------------------------------

@@ -668,6 +668,118 @@ def run_pipeline(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
             "plans": out, "iteration_time_reduction": 1.0 - best["iteration_ms"] / base["iteration_ms"]}
 
 
+class StageFwdRunner:
+    """Forward pass of one pipeline stage of 4 decoder layers built from the library's kernels: per layer
+    RMSNorm -> Q/K/V projections (K/V on owners) -> rotary embedding -> attention -> output projection ->
+    residual -> RMSNorm -> gate/up GEMMs -> SwiGLU -> down GEMM -> residual; the tail stage adds the final
+    norm and the LM head.  The operators run with the launch sequence and byte counts of a real forward pass
+    (layer l's kernels read layer l's own buffers rather than layer l-1's output, which does not change a
+    kernel's time)."""
+
+    def __init__(self, kvp, cfg, device, F=11008, V=32000, lm_head=False):
+        self.kvp, self.cfg, self.F, self.V, self.lm_head = kvp, cfg, F, V, lm_head
+        self.attn = TrainRunner(kvp, cfg, device, backward=False, out_proj=True, bucket=False)
+        bf = torch.bfloat16
+        T, D, L = cfg.T, cfg.D, cfg.L
+        rnd = lambda *shape: torch.randn(*shape, device=device, dtype=bf)
+        self.h = [rnd(T, D) for _ in range(L)]                     # residual stream entering each layer
+        self.wn1 = [rnd(D) for _ in range(L)]
+        self.wn2 = [rnd(D) for _ in range(L)]
+        self.w_gate = [rnd(F, D) * 0.02 for _ in range(L)]
+        self.w_up = [rnd(F, D) * 0.02 for _ in range(L)]
+        self.w_down = [rnd(D, F) * 0.02 for _ in range(L)]
+        self.gate, self.up = torch.empty(T, F, device=device, dtype=bf), torch.empty(T, F, device=device, dtype=bf)
+        self.mid = torch.empty(T, D, device=device, dtype=bf)
+        if lm_head:
+            self.w_lm = rnd(V, D) * 0.02
+            self.logits = torch.empty(T, V, device=device, dtype=bf)
+        self.elem_bytes = 0
+
+    def step(self, _i=0):
+        k, c, a = self.kvp, self.cfg, self.attn
+        t, o = a.t, a.out
+        own = set(c.owners())
+        eb = 0
+        T, D, F = c.T, c.D, self.F
+        for l in range(c.L):
+            k.rmsnorm(self.h[l], self.wn1[l], 1e-5, t["x"][l])
+            eb += 2 * T * D * 2
+        k.proj_fwd(a.sh, c.donor, t["x"], t["wq"], t["wk"], t["wv"], o["q"], o["k"], o["v"])
+        for l in range(c.L):
+            k.rope(o["q"][l])
+            eb += 2 * o["q"][l].numel() * 2
+            if l in own:
+                k.rope(o["k"][l])
+                eb += 2 * o["k"][l].numel() * 2
+        k.attn_fwd(a.sh, c.donor, o["q"], o["k"], o["v"], o["o"], o["lse"])
+        k.out_proj_fwd(a.sh, o["o"], t["wo"], o["y"])
+        for l in range(c.L):
+            k.add(self.h[l], o["y"][l], self.mid)
+            k.rmsnorm(self.mid, self.wn2[l], 1e-5, o["y"][l])
+            k.gemm(o["y"][l], self.w_gate[l], self.gate)
+            k.gemm(o["y"][l], self.w_up[l], self.up)
+            k.swiglu(self.gate, self.up, self.gate)
+            k.gemm(self.gate, self.w_down[l], o["y"][l])
+            k.add(self.mid, o["y"][l], self.mid)
+            eb += (3 + 2 + 3) * T * D * 2 + 3 * T * F * 2
+        if self.lm_head:
+            k.rmsnorm(self.mid, self.wn1[0], 1e-5, self.mid)
+            k.gemm(self.mid, self.w_lm, self.logits)
+            eb += 2 * T * D * 2
+        self.elem_bytes = eb
+
+
+def run_stage_fwd(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
+    """Whole-stage forward times (the paper's stage tables list one per stage): a regular stage, the tail stage
+    with the LM head, and the tail stage with three of its four layers converted (stage-local donor), LLaMA2-7B
+    geometry with MHA, S = 8192, one sequence per micro-batch."""
+    D, H, dh, S = 4096, 32, 128, 8192
+    full = W.TrainCfg("stage-mha-unconverted", 4, 1, S, D, H, H, dh, [0, 1, 2, 3])
+    local = W.TrainCfg("stage-mha-local-donor", 4, 1, S, D, H, H, dh, [0, 0, 0, 0])
+    res = {}
+    for name, cfg, lm in (("regular", full, False), ("tail", full, True), ("tail_converted", local, True)):
+        r = StageFwdRunner(kvp, cfg, device, lm_head=lm)
+        for i in range(max(args.warmup, 40)):       # long enough for the power-capped clock to settle
+            r.step(i)
+        ms, clocks = timed_region(r.step, args.steps, device, local_rank)
+        res[name] = {"ms": ms / args.steps, "elementwise_bytes": r.elem_bytes, "sm_mhz": clocks.get("sm_mhz")}
+        del r
+        torch.cuda.empty_cache()
+    # the element-wise kernels alone, against the measured copy bandwidth
+    r = StageFwdRunner(kvp, full, device)
+    T, F = full.T, r.F
+    def timed(fn, nbytes, reps=20):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        return {"us": us, "gbs": nbytes / (us * 1e-6) / 1e9, "frac_of_measured_copy": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+    q = r.attn.out["q"][0]
+    elem = {"rmsnorm": timed(lambda: kvp.rmsnorm(r.h[0], r.wn1[0], 1e-5, r.mid), 2 * T * D * 2),
+            "rope": timed(lambda: kvp.rope(q), 2 * q.numel() * 2),
+            "swiglu": timed(lambda: kvp.swiglu(r.gate, r.up, r.gate), 3 * T * F * 2),
+            "add": timed(lambda: kvp.add(r.h[0], r.h[1], r.mid), 3 * T * D * 2)}
+    del r
+    torch.cuda.empty_cache()
+    ff, fs, flm = kvp.layer_flops(D, 11008, H, H, dh, S, 32000)
+    return {"metric": "tail-stage forward ms (LLaMA2-7B MHA, S=8192, converted)", "value": res["tail_converted"]["ms"], "unit": "ms",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["tail_converted"]["ms"],
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "stage-forward-LLaMA2-7B-MHA-S8192", "layers_per_stage": 4, "tokens": S,
+                       "l2": "working set of a stage far larger than L2"},
+            "stages": res, "elementwise_kernels": elem,
+            "time_ratio_tail_over_regular": res["tail"]["ms"] / res["regular"]["ms"],
+            "time_ratio_converted_tail_over_regular": res["tail_converted"]["ms"] / res["regular"]["ms"],
+            "flops_ratio_tail_over_regular": (4 * ff + flm) / (4 * ff),
+            "flops_ratio_converted_tail_over_regular": (ff + 3 * fs + flm) / (4 * ff),
+            "device_status": kvp.status_string(kvp.device_status())}
+
+
 def reference_arm(args, rank, world):
     """The fp64 CPU oracle on this machine's host cores; each step is a bounded sample of the workload."""
     if rank != 0:
@@ -707,7 +819,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="train", choices=["train", "prefill", "decode", "stage", "pipeline", "decode_sweep"])
+    ap.add_argument("--workload", default="train", choices=["train", "prefill", "decode", "stage", "pipeline", "decode_sweep", "stage_fwd"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode workload in the default run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -742,6 +854,8 @@ def main():
             line["cpu_baseline"] = cpu_baseline_train(cfg, backward)
             if "decode" in line and "error" not in line["decode"]:
                 line["decode"]["cpu_baseline"] = cpu_baseline_decode(W.C3)
+    elif args.workload == "stage_fwd":
+        line = run_stage_fwd(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
     elif args.workload == "decode_sweep":
         line = run_decode_sweep(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
     elif args.workload == "pipeline":

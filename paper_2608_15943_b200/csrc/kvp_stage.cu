@@ -4,6 +4,8 @@
 // arithmetic, bf16 storage, one pass over the data, grids sized to the SM count.
 #include <math.h>
 
+#include <algorithm>
+
 #include "kvp_host.h"
 #include "kvp_sm100.cuh"
 
@@ -72,29 +74,40 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(const uint4* __re
 // In-place rotary embedding of x [B, S, H, dh]: pair i of every head turns by (pos0 + s) * theta^(-2i/dh).
 // One thread per 8 consecutive elements (4 pairs).  The frequencies arrive as float pairs hi + lo rounded from
 // the host's double values; the angle pos * f is formed as an exact product p = pos * hi plus its rounding
-// error and the lo term, sincosf(p) is exact for the float p at any magnitude, and the small remainder is
+// error and the lo term, sine and cosine of the float p are taken after an exact range reduction, and the small remainder is
 // applied as a second-order rotation (|remainder| <= half an ulp of p, below 2^-6 for the positions < 2^18
 // the entry point admits, so the neglected third-order term is under 1e-6).
 constexpr int kMaxRopePairs = 128;  // dh <= 256
 struct RopeFreq {
   float2 f[kMaxRopePairs];
 };
-__global__ void rope_kernel(uint4* __restrict__ x, size_t n8, int S, int H, int dh8, int pos0, const __grid_constant__ RopeFreq fr) {
-  const size_t stride = size_t(gridDim.x) * blockDim.x;
-  for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n8; i += stride) {
-    const int c = int(i % dh8);                       // which group of 4 pairs inside the head
-    const size_t tok = i / (size_t(dh8) * H);         // b * S + s
+__global__ void rope_kernel(uint4* __restrict__ x, uint32_t n8, uint32_t S, uint32_t per_tok, uint32_t dh8, int pos0,
+                            const __grid_constant__ RopeFreq fr) {
+  // lanes of a warp need different table entries: shared memory serves them in one pass, the constant bank
+  // that holds kernel parameters would replay once per distinct address
+  __shared__ float2 freq[kMaxRopePairs];
+  for (int k = threadIdx.x; k < kMaxRopePairs; k += blockDim.x) freq[k] = fr.f[k];
+  __syncthreads();
+  const uint32_t stride = gridDim.x * blockDim.x;
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {  // 32-bit index arithmetic only
+    const uint32_t c = i % dh8;                       // which group of 4 pairs inside the head
+    const uint32_t tok = i / per_tok;                 // b * S + s
     const float pos = float(pos0 + int(tok % S));     // exact
     float f[8];
     uint4 v = x[i];
     unpack8(v, f);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const float2 fq = fr.f[c * 4 + k];
+      const float2 fq = freq[c * 4 + k];
       const float p = pos * fq.x;
       const float d = fmaf(pos, fq.y, fmaf(pos, fq.x, -p));   // angle - p
-      float sn, cs;
-      sincosf(p, &sn, &cs);
+      // p (< 2^18) reduced to [-pi, pi] with 2*pi split into three floats whose first has 8 significant
+      // bits, so that k * 6.28125 is exact and the subtraction loses nothing (error about 1e-7)
+      const float kk = rintf(p * 0.15915494309189535f);
+      float rr = fmaf(-kk, 6.28125f, p);
+      rr = fmaf(-kk, 0.00193023681640625f, rr);
+      rr = fmaf(-kk, 5.070363386039389e-06f, rr);
+      const float sn = __sinf(rr), cs = __cosf(rr);
       const float h = 0.5f * d * d;
       const float sn2 = sn + d * cs - h * sn, cs2 = cs - d * sn - h * cs;
       const float a = f[2 * k], b = f[2 * k + 1];
@@ -113,7 +126,7 @@ __global__ void swiglu_kernel(const uint4* __restrict__ gate, const uint4* __res
     unpack8(gate[i], g);
     unpack8(up[i], u);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) g[k] = g[k] / (1.f + __expf(-g[k])) * u[k];
+    for (int k = 0; k < 8; ++k) g[k] = g[k] * __frcp_rn(1.f + __expf(-g[k])) * u[k];
     out[i] = pack8(g);
   }
 }
@@ -160,9 +173,16 @@ extern "C" int kvp_rope(int32_t B, int32_t S, int32_t H, int32_t dh, float theta
     fr.f[i].x = float(f);
     fr.f[i].y = float(f - double(fr.f[i].x));
   }
-  rope_kernel<<<streaming_blocks(n8, 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(reinterpret_cast<uint4*>(x), n8, S, H,
-                                                                                              dh / 8, pos0, fr);
-  note_launch();
+  // 16-byte groups are indexed with 32 bits: larger tensors go in slices of whole sequences
+  const size_t per_seq = size_t(S) * H * (dh / 8);
+  if (per_seq >= (size_t(1) << 31)) return KVP_ERR_UNSUPPORTED;
+  const int seqs_per_launch = int(std::max<size_t>(1, ((size_t(1) << 31) - 1) / per_seq));
+  for (int b0 = 0; b0 < B; b0 += seqs_per_launch) {
+    const uint32_t m8 = uint32_t(size_t(std::min(seqs_per_launch, B - b0)) * per_seq);
+    rope_kernel<<<streaming_blocks(m8, 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<uint4*>(x) + size_t(b0) * per_seq, m8, uint32_t(S), uint32_t(H) * (dh / 8), uint32_t(dh / 8), pos0, fr);
+    note_launch();
+  }
   return cudaGetLastError() == cudaSuccess ? KVP_OK : KVP_ERR_CUDA;
 }
 

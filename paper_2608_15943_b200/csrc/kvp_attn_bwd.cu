@@ -762,35 +762,55 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
   }
 }
 
-// Delta[b,hq,s] = sum_c dO[b,s,hq,c] * O[b,s,hq,c]; one warp per (token, head) row.
+// Delta[b,hq,s] = sum_c dO[b,s,hq,c] * O[b,s,hq,c].  A row of DH bf16 is DH/8 16-byte pieces: each warp takes
+// 256/DH rows at a time (one piece per lane, every lane busy), two such groups per iteration so that four
+// loads per lane are in flight, and reduces inside the DH/8-lane segments.
 template <int DH>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                              float* __restrict__ delta, int B, int S, int Hq) {
+  constexpr int LANES = DH / 8;          // lanes per row
+  constexpr int ROWS = 32 / LANES;       // rows per warp and load
   const size_t rows = size_t(B) * S * Hq;
   const int lane = threadIdx.x & 31;
+  const int sub = lane / LANES, piece = lane % LANES;
   const size_t warp_global = (size_t(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
   const size_t n_warps = (size_t(gridDim.x) * blockDim.x) >> 5;
-  for (size_t row = warp_global; row < rows; row += n_warps) {
+  auto dot8 = [](const uint4& a, const uint4& g) {
+    const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g);
     float acc = 0.f;
-    if (lane * 8 < DH) {  // DH/8 lanes each take 16 bytes
-      const uint4 a = *reinterpret_cast<const uint4*>(o + row * DH + lane * 8);
-      const uint4 g = *reinterpret_cast<const uint4*>(d_o + row * DH + lane * 8);
-      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
-      const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 fa = __bfloat1622float2(pa[i]), fg = __bfloat1622float2(pg[i]);
-        acc += fa.x * fg.x + fa.y * fg.y;
-      }
+    for (int i = 0; i < 4; ++i) {
+      const float2 fa = __bfloat1622float2(pa[i]), fg = __bfloat1622float2(pg[i]);
+      acc += fa.x * fg.x + fa.y * fg.y;
     }
+    return acc;
+  };
+  for (size_t base = warp_global * (2 * ROWS); base < rows; base += n_warps * (2 * ROWS)) {
+    const size_t r0 = base + sub, r1 = base + ROWS + sub;
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    const uint4 a0 = r0 < rows ? *reinterpret_cast<const uint4*>(o + r0 * DH + piece * 8) : z;
+    const uint4 g0 = r0 < rows ? *reinterpret_cast<const uint4*>(d_o + r0 * DH + piece * 8) : z;
+    const uint4 a1 = r1 < rows ? *reinterpret_cast<const uint4*>(o + r1 * DH + piece * 8) : z;
+    const uint4 g1 = r1 < rows ? *reinterpret_cast<const uint4*>(d_o + r1 * DH + piece * 8) : z;
+    float acc0 = dot8(a0, g0), acc1 = dot8(a1, g1);
 #pragma unroll
-    for (int sft = 16; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
-    if (lane == 0) {
-      const int hq = int(row % Hq);
-      const size_t tok = row / Hq;
-      const int s = int(tok % S);
-      const int b = int(tok / S);
-      delta[(size_t(b) * Hq + hq) * S + s] = acc;
+    for (int sft = LANES / 2; sft > 0; sft >>= 1) {
+      acc0 += __shfl_xor_sync(0xffffffffu, acc0, sft);
+      acc1 += __shfl_xor_sync(0xffffffffu, acc1, sft);
+    }
+    if (piece == 0) {
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const size_t row = u == 0 ? r0 : r1;
+        if (row < rows) {
+          const int hq = int(row % Hq);
+          const size_t tok = row / Hq;
+          const int sx = int(tok % S);
+          const int bx = int(tok / S);
+          delta[(size_t(bx) * Hq + hq) * S + sx] = u == 0 ? acc0 : acc1;
+        }
+      }
     }
   }
 }

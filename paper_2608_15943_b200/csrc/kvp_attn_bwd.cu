@@ -192,14 +192,15 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      tma_prefetch_desc(&p.map_k);
-      tma_prefetch_desc(&p.map_v);
-      mbar_expect_tx(kv_full, 2 * L::KV_TILE);
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
+      if (leader) tma_prefetch_desc(&p.map_k);
+      if (leader) tma_prefetch_desc(&p.map_v);
+      mbar_expect_tx_e(kv_full, 2 * L::KV_TILE, leader);
 #pragma unroll
       for (int h = 0; h < HALVES; ++h) {
-        tma_load_4d(smem + L::OFF_K + h * HALF_BYTES, &p.map_k, kv_full, h * 64, hk, kv0, b);
-        tma_load_4d(smem + L::OFF_V + h * HALF_BYTES, &p.map_v, kv_full, h * 64, hk, kv0, b);
+        tma_load_4d_e(smem + L::OFF_K + h * HALF_BYTES, &p.map_k, kv_full, h * 64, hk, kv0, b, leader);
+        tma_load_4d_e(smem + L::OFF_V + h * HALF_BYTES, &p.map_v, kv_full, h * 64, hk, kv0, b, leader);
       }
       for (int it = 0; it < n_iter; ++it) {
         int li, hq, q0;
@@ -207,12 +208,12 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         const int s = it % DKDV_STAGES;
         const uint32_t ph = (it / DKDV_STAGES) & 1;
         if (!mbar_wait(&q_empty[s], ph ^ 1, err)) break;
-        mbar_expect_tx(&q_full[s], L::STAGE);
+        mbar_expect_tx_e(&q_full[s], L::STAGE, leader);
         uint8_t* dst = smem + L::OFF_RING + s * L::STAGE;
 #pragma unroll
         for (int h = 0; h < HALVES; ++h) {
-          tma_load_4d(dst + h * QHALF_BYTES, &p.map_q[li], &q_full[s], h * 64, hq, q0, b);
-          tma_load_4d(dst + L::Q_TILE + h * QHALF_BYTES, &p.map_do[li], &q_full[s], h * 64, hq, q0, b);
+          tma_load_4d_e(dst + h * QHALF_BYTES, &p.map_q[li], &q_full[s], h * 64, hq, q0, b, leader);
+          tma_load_4d_e(dst + L::Q_TILE + h * QHALF_BYTES, &p.map_do[li], &q_full[s], h * 64, hq, q0, b, leader);
         }
       }
     }
@@ -541,34 +542,35 @@ __global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      tma_prefetch_desc(&p.map_q);
-      tma_prefetch_desc(&p.map_do);
-      tma_prefetch_desc(&p.map_k);
-      tma_prefetch_desc(&p.map_v);
-      mbar_expect_tx(qdo_full, 4 * L::TILE);  // rows beyond the sequence are zero-filled
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
+      if (leader) tma_prefetch_desc(&p.map_q);
+      if (leader) tma_prefetch_desc(&p.map_do);
+      if (leader) tma_prefetch_desc(&p.map_k);
+      if (leader) tma_prefetch_desc(&p.map_v);
+      mbar_expect_tx_e(qdo_full, 4 * L::TILE, leader);  // rows beyond the sequence are zero-filled
 #pragma unroll
       for (int x = 0; x < 2; ++x)
 #pragma unroll
         for (int h = 0; h < HALVES; ++h) {
-          tma_load_4d(smem + L::OFF_Q + x * L::TILE + h * HALF_BYTES, &p.map_q, qdo_full, h * 64, hq, q0 + x * BT, b);
-          tma_load_4d(smem + L::OFF_DO + x * L::TILE + h * HALF_BYTES, &p.map_do, qdo_full, h * 64, hq, q0 + x * BT, b);
+          tma_load_4d_e(smem + L::OFF_Q + x * L::TILE + h * HALF_BYTES, &p.map_q, qdo_full, h * 64, hq, q0 + x * BT, b, leader);
+          tma_load_4d_e(smem + L::OFF_DO + x * L::TILE + h * HALF_BYTES, &p.map_do, qdo_full, h * 64, hq, q0 + x * BT, b, leader);
         }
       auto load_k = [&](int j) -> bool {
         const int s = j % DQ_KSTAGES;
         if (!mbar_wait(&k_empty[s], ((j / DQ_KSTAGES) & 1) ^ 1, err)) return false;
-        mbar_expect_tx(&k_full[s], L::TILE);
+        mbar_expect_tx_e(&k_full[s], L::TILE, leader);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_K + s * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BT, b);
+          tma_load_4d_e(smem + L::OFF_K + s * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BT, b, leader);
         return true;
       };
       auto load_v = [&](int j) -> bool {
         if (!mbar_wait(v_empty, (j & 1) ^ 1, err)) return false;
-        mbar_expect_tx(v_full, L::TILE);
+        mbar_expect_tx_e(v_full, L::TILE, leader);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_V + h * HALF_BYTES, &p.map_v, v_full, h * 64, hk, j * BT, b);
+          tma_load_4d_e(smem + L::OFF_V + h * HALF_BYTES, &p.map_v, v_full, h * 64, hk, j * BT, b, leader);
         return true;
       };
       bool ok = n_max > 0 ? load_k(0) : true;

@@ -124,32 +124,33 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      tma_prefetch_desc(&p.map_q);
-      tma_prefetch_desc(&p.map_k);
-      tma_prefetch_desc(&p.map_v);
-      mbar_expect_tx(q_full, 2 * L::Q_BYTES);  // rows beyond the sequence are zero-filled
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
+      if (leader) tma_prefetch_desc(&p.map_q);
+      if (leader) tma_prefetch_desc(&p.map_k);
+      if (leader) tma_prefetch_desc(&p.map_v);
+      mbar_expect_tx_e(q_full, 2 * L::Q_BYTES, leader);  // rows beyond the sequence are zero-filled
 #pragma unroll
       for (int x = 0; x < 2; ++x)
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_Q + x * L::Q_BYTES + h * HALF_BYTES, &p.map_q, q_full, h * 64, hq, q0 + x * BQ, b);
+          tma_load_4d_e(smem + L::OFF_Q + x * L::Q_BYTES + h * HALF_BYTES, &p.map_q, q_full, h * 64, hq, q0 + x * BQ, b, leader);
       auto load_k = [&](int j) -> bool {
         const int s = j % FWD_KSTAGES;
         if (!mbar_wait(&k_empty[s], ((j / FWD_KSTAGES) & 1) ^ 1, err)) return false;
-        mbar_expect_tx(&k_full[s], L::KV_BYTES);
+        mbar_expect_tx_e(&k_full[s], L::KV_BYTES, leader);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_K + s * L::KV_BYTES + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BKV, b);
+          tma_load_4d_e(smem + L::OFF_K + s * L::KV_BYTES + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BKV, b, leader);
         return true;
       };
       auto load_v = [&](int j) -> bool {
         const int s = j % FWD_VSTAGES;
         if (!mbar_wait(&v_empty[s], ((j / FWD_VSTAGES) & 1) ^ 1, err)) return false;
-        mbar_expect_tx(&v_full[s], L::KV_BYTES);
+        mbar_expect_tx_e(&v_full[s], L::KV_BYTES, leader);
 #pragma unroll
         for (int h = 0; h < HALVES; ++h)
-          tma_load_4d(smem + L::OFF_V + s * L::KV_BYTES + h * HALF_BYTES, &p.map_v, &v_full[s], h * 64, hk, j * BKV, b);
+          tma_load_4d_e(smem + L::OFF_V + s * L::KV_BYTES + h * HALF_BYTES, &p.map_v, &v_full[s], h * 64, hk, j * BKV, b, leader);
         return true;
       };
       bool ok = n_max > 0 ? load_k(0) : true;

@@ -89,11 +89,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      for (int s = 0; s < p.nseg; ++s) {
-        tma_prefetch_desc(&p.map_a[s]);
-        tma_prefetch_desc(&p.map_b[s]);
-      }
+    {
+      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
+      if (lane == 0)
+        for (int s = 0; s < p.nseg; ++s) {
+          tma_prefetch_desc(&p.map_a[s]);
+          tma_prefetch_desc(&p.map_b[s]);
+        }
+      __syncwarp();
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
@@ -107,19 +110,19 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
             if (!mbar_wait(&empty[s], ph ^ 1, err)) { ok = false; break; }
             uint8_t* sa = smem + size_t(s) * STAGE_BYTES;
             uint8_t* sb = sa + A_BYTES;
-            mbar_expect_tx(&full[s], STAGE_BYTES);
+            mbar_expect_tx_e(&full[s], STAGE_BYTES, leader);
             const int k0 = kb * BK;
             if (p.a_mn == 0) {
-              tma_load_2d(sa, &p.map_a[seg], &full[s], k0, m0);
+              tma_load_2d_e(sa, &p.map_a[seg], &full[s], k0, m0, leader);
             } else {
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * 8192, &p.map_a[seg], &full[s], m0 + 64 * j, k0);
+              for (int j = 0; j < BM / 64; ++j) tma_load_2d_e(sa + j * 8192, &p.map_a[seg], &full[s], m0 + 64 * j, k0, leader);
             }
             if (p.b_mn == 0) {
-              tma_load_2d(sb, &p.map_b[seg], &full[s], k0, n0);
+              tma_load_2d_e(sb, &p.map_b[seg], &full[s], k0, n0, leader);
             } else {
 #pragma unroll
-              for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, &p.map_b[seg], &full[s], n0 + 64 * j, k0);
+              for (int j = 0; j < BN / 64; ++j) tma_load_2d_e(sb + j * 8192, &p.map_b[seg], &full[s], n0 + 64 * j, k0, leader);
             }
           }
         }

@@ -103,6 +103,39 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, u
       "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
       : "memory");
 }
+// Elected-lane forms for a producer warp that runs its loop converged (see elect_one below): `leader` is
+// nonzero in exactly one lane.
+__device__ __forceinline__ void mbar_expect_tx_e(uint64_t* bar, uint32_t bytes, uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred q;\n"
+      " setp.ne.b32 q, %2, 0;\n"
+      " @q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n"
+      "}\n" ::"r"(smem_u32(bar)),
+      "r"(bytes), "r"(leader)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_e(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y, uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred q;\n"
+      " setp.ne.b32 q, %5, 0;\n"
+      " @q cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+      "}\n" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(leader)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_e(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z, int w,
+                                              uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred q;\n"
+      " setp.ne.b32 q, %7, 0;\n"
+      " @q cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+      "}\n" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(leader)
+      : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map),
                "r"(smem_u32(src)), "r"(x), "r"(y)

@@ -37,7 +37,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one-pass ncu captures of the
 # full-size launches, averaged over the launches of one step; summary and commands in profiles/traffic_full-size.md.
-NCU_TRAFFIC_BYTES = {"dkdv_kernel": 1.627e9, "dq_kernel": 0.664e9, "attn_fwd_kernel": 0.471e9, "decode_kernel": 77.96e9}
+NCU_TRAFFIC_BYTES = {"dkdv_kernel": 1.663e9, "dq_kernel": 0.663e9, "attn_fwd_kernel": 0.474e9, "decode_kernel": 77.96e9}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -35,9 +35,11 @@ from paper_2608_15943_b200 import workloads as W          # noqa: E402
 
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one-pass ncu captures of the
-# full-size launches, averaged over the launches of one step; summary and commands in profiles/traffic_full-size.md.
-NCU_TRAFFIC_BYTES = {"dkdv_kernel": 1.663e9, "dq_kernel": 0.663e9, "attn_fwd_kernel": 0.474e9, "decode_kernel": 77.96e9}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum): STORED CONSTANTS, not measured by this
+# program.  They come from ncu captures of the small case of each kernel, scaled to a full-size launch by the units
+# one launch processes (traffic grows in proportion); the committed profile summaries give the captures and dates.
+NCU_TRAFFIC_BYTES = {"bwd_kernel": None, "attn_fwd_kernel": 0.474e9, "decode_kernel": 77.96e9}
+NCU_TRAFFIC_NOTE = "bytes per launch; a stored constant from an earlier ncu capture, not measured in this run"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -181,20 +183,52 @@ class TrainRunner:
         f = c.proj_fwd_flops() + (c.L * 2 * c.T * c.D * c.Hq * c.dh if self.out_proj else 0)
         return 3 * f if self.backward else f
 
-    # End to end: every step's inputs come from pinned host memory and the block's dX goes back.  The copies
-    # are pipelined the way an input loader does it: while step n computes, a second stream brings step
-    # n+1's inputs into the other of two device buffer sets, and a third takes step n's result out.  Every
-    # call issues exactly one input copy and one result copy and does not return the compute stream until
-    # the input copy it issued has landed, so K timed calls contain K input and K result transfers.
-    def setup_e2e(self):
-        names = ["x", "dy" if self.out_proj else "d_o"] if self.backward else ["x"]
-        self.e2e_names = names
-        self.h_in = {n: [a.cpu().pin_memory() for a in self.t[n]] for n in names}
-        self.in_sets = [{n: self.t[n] for n in names}, {n: [torch.empty_like(a) for a in self.t[n]] for n in names}]
-        self.h_out = torch.empty_like(self.out["dx"][0] if self.backward else self.out["o"][-1],
-                                      device="cpu").pin_memory()
-        self.h2d = sum(a.numel() * a.element_size() for n in names for a in self.h_in[n])
-        self.d2h = self.h_out.numel() * self.h_out.element_size()
+    def attn_step(self, ins, before_results=None):
+        """Attention only (the headline metric's unit of work): forward, then backward, on the q / k / v / dO given."""
+        k, c, o = self.kvp, self.cfg, self.out
+        if not self.backward and before_results is not None:
+            before_results()
+        k.attn_fwd(self.sh, c.donor, ins["q"], ins["k"], ins["v"], o["o"], o["lse"])
+        if self.backward:
+            if before_results is not None:
+                before_results()
+            k.attn_bwd(self.sh, c.donor, ins["q"], ins["k"], ins["v"], o["o"], ins["d_o"], o["lse"], o["dq"], o["dk_sum"],
+                       o["dv_sum"], self.ws)
+
+    # End to end: every step's inputs come from pinned host memory and its results go back to pinned host memory.
+    #   mode "attn":  q, k, v (and dO) in; O (forward only) or dQ, dK/dV sums (with backward) out -- the calls a user
+    #                 of kvp_attn_fwd / kvp_attn_bwd with host-resident tensors makes;
+    #   mode "block": X (and dO) in; O of every layer (forward only) or dX of every layer and the whole weight-gradient
+    #                 bucket (with backward) out.
+    # The copies are pipelined the way an input loader does it: while step n computes, a second stream brings step
+    # n+1's inputs into the other of two device buffer sets, and a third takes step n's results out.  Every call
+    # issues exactly one input copy and one result copy and does not return the compute stream until the input
+    # copy it issued has landed, so K timed calls contain K input and K result transfers.
+    def setup_e2e(self, mode):
+        o, t = self.out, self.t
+        self.e2e_mode = mode
+        if mode == "attn":
+            self.step()                          # q, k, v of this batch
+            torch.cuda.synchronize()
+            cur_in = {"q": o["q"], "k": o["k"], "v": o["v"]}
+            if self.backward:
+                cur_in["d_o"] = t["d_o"]
+            results = (o["dq"] + [x for x in o["dk_sum"] if x is not None] + [x for x in o["dv_sum"] if x is not None]) \
+                if self.backward else list(o["o"])
+        else:
+            cur_in = {"x": t["x"]}
+            if self.backward:
+                cur_in["dy" if self.out_proj else "d_o"] = t["dy" if self.out_proj else "d_o"]
+            results = (list(o["dx"]) + ([self.bucket.flat] if self.bucket is not None else [])) if self.backward \
+                else list(o["o"])
+        dup = lambda xs: [None if a is None else torch.empty_like(a) for a in xs]
+        self.in_sets = [cur_in, {n: dup(xs) for n, xs in cur_in.items()}]
+        self.h_in = {n: [None if a is None else a.cpu().pin_memory() for a in xs] for n, xs in cur_in.items()}
+        self.results = results
+        self.h_out = [torch.empty_like(a, device="cpu").pin_memory() for a in results]
+        nb = lambda xs: sum(a.numel() * a.element_size() for a in xs if a is not None)
+        self.h2d = sum(nb(xs) for xs in self.h_in.values())
+        self.d2h = nb(self.h_out)
         self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
         self.ev_in = [torch.cuda.Event(), torch.cuda.Event()]      # input set filled
         self.ev_free = [torch.cuda.Event(), torch.cuda.Event()]    # input set no longer read
@@ -209,35 +243,48 @@ class TrainRunner:
         with torch.cuda.stream(self.s_in):
             if after is not None:
                 self.s_in.wait_event(after)    # the set's previous reader has finished
-            for n in self.e2e_names:
-                for dst, src in zip(self.in_sets[which][n], self.h_in[n]):
-                    dst.copy_(src, non_blocking=True)
+            for n, hs in self.h_in.items():
+                for dst, src in zip(self.in_sets[which][n], hs):
+                    if dst is not None:
+                        dst.copy_(src, non_blocking=True)
             self.ev_in[which].record(self.s_in)
 
     def step_e2e(self, _i=0):
         cur = torch.cuda.current_stream()
         a = self.e2e_calls & 1
         self.e2e_calls += 1
-        for n in self.e2e_names:
-            self.t[n] = self.in_sets[a][n]
+        ins = self.in_sets[a]
         # next step's inputs into the other set, once the step before this one has stopped reading it
         self._copy_in(1 - a, after=self.ev_free[1 - a] if self.e2e_calls > 1 else None)
-        result = self.out["dx"][0] if self.backward else self.out["o"][-1]
-        # the previous result must have left the device before this step overwrites it
-        if self.backward:
-            self.step(before_proj_bwd=lambda: cur.wait_event(self.ev_out))
+        # the previous results must have left the device before this step overwrites them
+        wait_out = lambda: cur.wait_event(self.ev_out)
+        if self.e2e_mode == "attn":
+            self.attn_step(ins, before_results=wait_out)
         else:
-            cur.wait_event(self.ev_out)
-            self.step()
+            for n, xs in ins.items():
+                self.t[n] = xs
+            if self.backward:
+                self.step(before_proj_bwd=wait_out)
+            else:
+                wait_out()
+                self.step()
         self.ev_free[a].record(cur)
         self.ev_result.record(cur)
         with torch.cuda.stream(self.s_out):
             self.s_out.wait_event(self.ev_result)
-            self.h_out.copy_(result, non_blocking=True)
+            for dst, src in zip(self.h_out, self.results):
+                dst.copy_(src, non_blocking=True)
             self.ev_out.record(self.s_out)
         cur.wait_event(self.ev_in[1 - a])      # the copy issued by this call is inside this call's time
         if _i == getattr(self, "e2e_last", -1):  # the last timed call also waits for its own result copy
             cur.wait_event(self.ev_out)
+
+    def teardown_e2e(self):
+        torch.cuda.synchronize()
+        for n in ("in_sets", "h_in", "h_out", "results"):
+            if hasattr(self, n):
+                delattr(self, n)
+        torch.cuda.empty_cache()
 
 
 def cpu_baseline_train(cfg: W.TrainCfg, backward: bool, heads: int = 4, proj_tokens: int = 1024):
@@ -258,33 +305,38 @@ def cpu_baseline_train(cfg: W.TrainCfg, backward: bool, heads: int = 4, proj_tok
     wv = [synth.normal((nkv, D), seed, synth.tid(3), 0.02).double().numpy()]
     t0 = time.perf_counter()
     A.attn_fwd(q, k, v, [0])
-    qq, kk, vv = A.proj_fwd(x, wq, wk, wv, [0], 1, proj_tokens, cfg.Hq, cfg.Hkv, dh)
     if backward:
         A.attn_bwd(q, k, v, g, [0])
+    dt_attn = time.perf_counter() - t0
+    qq, kk, vv = A.proj_fwd(x, wq, wk, wv, [0], 1, proj_tokens, cfg.Hq, cfg.Hkv, dh)
+    if backward:
         A.proj_bwd(x, wq, wk, wv, qq, kk, vv, [0])
     dt = time.perf_counter() - t0
-    flops = 4 * dh * (S * (S + 1) // 2) * heads + 2 * proj_tokens * D * (nq + 2 * nkv)
+    f_attn = 4 * dh * (S * (S + 1) // 2) * heads
+    f_proj = 2 * proj_tokens * D * (nq + 2 * nkv)
     if backward:
-        flops *= 3
+        f_attn, f_proj = 3 * f_attn, 3 * f_proj
     try:
         from threadpoolctl import threadpool_info
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
         cores = os.cpu_count() or 1
     sample = (f"attention fwd{'+bwd' if backward else ''} of 1 layer x 1 sequence x {heads} query heads (one KV group) "
-              f"at S={S}, plus Q/K/V projections fwd{'+bwd' if backward else ''} of one owner layer on {proj_tokens} tokens; "
-              f"{flops / 1e9:.1f} model GFLOP in {dt:.2f} s")
-    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
-            "seconds": dt}
+              f"at S={S}: {f_attn / 1e9:.1f} model GFLOP in {dt_attn:.2f} s (the value); plus Q/K/V projections "
+              f"fwd{'+bwd' if backward else ''} of one owner layer on {proj_tokens} tokens: {f_proj / 1e9:.1f} GFLOP in {dt - dt_attn:.2f} s")
+    return {"value": f_attn / dt_attn / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
+            "seconds": dt, "block_value": (f_attn + f_proj) / dt / 1e12}
 
 
 # ---------------------------------------------------------------------------------------------
 # decode workload
 # ---------------------------------------------------------------------------------------------
 class DecodeRunner:
-    def __init__(self, kvp, cfg: W.DecodeCfg, device, n_slots=None, q_sets=4):
-        self.kvp, self.cfg, self.device = kvp, cfg, device
-        self.state = W.make_decode_state(cfg, device, n_slots=n_slots)
+    def __init__(self, kvp, cfg: W.DecodeCfg, device, n_slots=None, q_sets=4, shuffle_pages=True, per_layer=False):
+        """per_layer: one kvp_decode call per layer (layer_begin / layer_end), the order a real model's forward
+        pass imposes -- a consumer then re-reads its donor's pages -- instead of one grouped call per step."""
+        self.kvp, self.cfg, self.device, self.per_layer = kvp, cfg, device, per_layer
+        self.state = W.make_decode_state(cfg, device, n_slots=n_slots, shuffle_pages=shuffle_pages)
         st = self.state
         self.desc = kvp.DecodeDesc(cfg.L, cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, cfg.page, cfg.max_pages, st.n_pages, 0)
         self.ws = torch.empty(kvp.decode_workspace_bytes(self.desc, cfg.donor), dtype=torch.uint8, device=device)
@@ -308,8 +360,13 @@ class DecodeRunner:
         st.lengths.add_(1)                       # the new token is part of the context it attends to
         k.cache_append(self.desc, c.donor, self.k_new[s], self.v_new[s], st.k_cache, st.v_cache, st.block_table,
                        st.lengths)
-        k.decode(self.desc, c.donor, self.q[s], st.k_cache, st.v_cache, st.block_table, st.lengths, self.o,
-                 self.lse, self.ws)
+        if self.per_layer:
+            for l in range(c.L):
+                k.decode(self.desc, c.donor, self.q[s], st.k_cache, st.v_cache, st.block_table, st.lengths, self.o,
+                         self.lse, self.ws, layer_begin=l, layer_end=l + 1)
+        else:
+            k.decode(self.desc, c.donor, self.q[s], st.k_cache, st.v_cache, st.block_table, st.lengths, self.o,
+                     self.lse, self.ws)
         self.steps_done += 1
 
     def setup_e2e(self):
@@ -359,13 +416,18 @@ def cpu_baseline_decode(cfg: W.DecodeCfg, n_seq: int = 16):
 
 
 # ---------------------------------------------------------------------------------------------
-def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind):
-    if args.workload == "train":
+def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, workload=None, e2e=True):
+    """Times the block step (projections + attention, forward [+ backward]) of C2 / C1 and reports, as `value`,
+    the ATTENTION-ONLY rate: model FLOPs of the attention kernels (12 dh pairs B Hq per layer with backward, 4 dh
+    pairs B Hq forward only, pairs = S(S+1)/2) over the summed device time of those kernels (forward, backward,
+    and the backward's helper passes) inside the timed region.  The block rate is reported beside it."""
+    workload = workload or args.workload
+    if workload == "train":
         cfg, backward, out_proj = (W.SMALL_TRAIN if args.small else W.C2), True, False
-    elif args.workload == "prefill":
+    elif workload == "prefill":
         cfg, backward, out_proj = (W.SMALL_TRAIN if args.small else W.C1), False, False
     else:
-        raise ValueError(args.workload)
+        raise ValueError(workload)
     runner = TrainRunner(kvp, cfg, device, backward=backward, out_proj=out_proj)
     for i in range(args.warmup):
         runner.step(i)
@@ -377,13 +439,14 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
     pairs = cfg.S * (cfg.S + 1) // 2
     unit = 2 * cfg.dh * pairs * cfg.B * cfg.Hq * cfg.L        # one attention GEMM over every layer
     n_gemm = (cfg.L + 2 * n_own) + ((2 * cfg.L + 2 * n_own) if backward else 0)
-    # kernel -> (launches per step, algorithmic FLOPs per step, executed FLOPs per step)
+    # kernel -> (timed event pairs per step, algorithmic FLOPs per step, executed FLOPs per step)
     kernels = {"attn_fwd_kernel": (kvp.KERNEL_ATTN_FWD, cfg.L, 2 * unit, 2 * unit),
                "gemm_kernel": (kvp.KERNEL_GEMM, n_gemm, runner.gemm_flops(), runner.gemm_flops())}
     if backward:
-        # dK/dV kernel: dV, dP, dK of the model count (it also recomputes S); dQ kernel: dQ (recomputes S, dP)
-        kernels["dkdv_kernel"] = (kvp.KERNEL_ATTN_BWD, n_groups, 3 * unit, 4 * unit)
-        kernels["dq_kernel"] = (kvp.KERNEL_ATTN_BWD_DQ, cfg.L, 1 * unit, 3 * unit)
+        # single-pass backward: dV, dP, dK, dQ of the model count (it also recomputes S); helper passes: Delta,
+        # clearing the fp32 accumulators, converting dQ to bf16 (no FLOPs counted)
+        kernels["bwd_kernel"] = (kvp.KERNEL_ATTN_BWD, n_groups, 4 * unit, 5 * unit)
+        kernels["bwd_aux"] = (kvp.KERNEL_ATTN_BWD_AUX, 1 + 2 * n_groups, 0, 0)
     timers = {name: kvp.KernelTimer(kid, args.steps * n) for name, (kid, n, _a, _e) in kernels.items()}
     l0 = kvp.launch_count()
     for t in timers.values():
@@ -394,38 +457,61 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
     launches = kvp.launch_count() - l0
     ms_step = ms / args.steps
     flops = runner.flops()
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    block_tflops = world * flops / (ms_step * 1e-3) / 1e12
     peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
     per_kernel = {}
     for name, (kid, n, algo, execd) in kernels.items():
         k_ms = sum(timers[name].durations_ms()) / args.steps
-        per_kernel[name] = {"launches_per_step": n, "ms_per_step": k_ms, "share_of_step": k_ms / ms_step,
+        per_kernel[name] = {"timed_launch_groups_per_step": n, "ms_per_step": k_ms, "share_of_step": k_ms / ms_step,
                             "algorithmic_tflops": algo / (k_ms * 1e-3) / 1e12,
                             "executed_tflops": execd / (k_ms * 1e-3) / 1e12}
-    top = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_step"])
+    attn_names = [n for n in per_kernel if n != "gemm_kernel"]
+    attn_ms = kdist.max_over_ranks(sum(per_kernel[n]["ms_per_step"] for n in attn_names), device)
+    attn_units = 6 if backward else 2
+    value = world * attn_units * unit / (attn_ms * 1e-3) / 1e12
+    flash = world * (7 if backward else 2) * unit / (attn_ms * 1e-3) / 1e12
+    top = max((n for n in per_kernel if n != "bwd_aux"), key=lambda k: per_kernel[k]["ms_per_step"])
     achieved = per_kernel[top]["algorithmic_tflops"]
+    traffic = None if args.small or cfg is not W.C2 else NCU_TRAFFIC_BYTES.get(top)
     roofline = {"bound": "tensor", "kernel": top + "<128>", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak,
-                "traffic": None if args.small or cfg is not W.C2 else NCU_TRAFFIC_BYTES.get(top),
-                "traffic_unit": "bytes per launch (ncu, full-size capture)",
+                "frac": achieved / peak, "traffic": traffic,
+                "traffic_unit": NCU_TRAFFIC_NOTE,
                 "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
-                "launches_per_step": per_kernel[top]["launches_per_step"],
+                "launches_per_step": n_groups if top == "bwd_kernel" else per_kernel[top]["timed_launch_groups_per_step"],
                 "kernel_ms_per_step": per_kernel[top]["ms_per_step"],
                 "share_of_step": per_kernel[top]["share_of_step"],
                 "executed_tflops": per_kernel[top]["executed_tflops"],
                 "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS, "kernels": per_kernel}
     # end to end through the public API with host buffers
-    if args.small:      # profiler capture: the device-timed region is all that is needed
-        ms_e2e, e2e_steps, e2e_val = float("nan"), 1, float("nan")
-        runner.h2d = runner.d2h = 0
-    else:
-        runner.setup_e2e()
-        for i in range(2):
-            runner.step_e2e(i)
+    e2e_obj, block_e2e = None, None
+    if e2e and not args.small:
         e2e_steps = max(3, min(args.steps, 5))
-        runner.e2e_last = e2e_steps - 1
-        ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
-        e2e_val = world * flops / (ms_e2e / e2e_steps * 1e-3) / 1e12
+        for mode in ("attn", "block"):
+            runner.setup_e2e(mode)
+            for i in range(2):
+                runner.step_e2e(i)
+            runner.e2e_last = e2e_steps - 1 + 2
+            calls0 = runner.e2e_calls
+            ms_e2e, _ = timed_region(lambda i: runner.step_e2e(i + 2), e2e_steps, device, local_rank)
+            assert runner.e2e_calls - calls0 == e2e_steps
+            f = (attn_units * unit) if mode == "attn" else flops
+            obj = {"value": world * f / (ms_e2e / e2e_steps * 1e-3) / 1e12, "unit": "TFLOP/s",
+                   "h2d_bytes_per_step": runner.h2d, "d2h_bytes_per_step": runner.d2h, "ms_per_step": ms_e2e / e2e_steps,
+                   "copies": "pipelined: step n+1's inputs arrive on a second stream while step n computes; "
+                             "one input and one result transfer per timed step"}
+            if mode == "attn":
+                obj["what"] = ("kvp_attn_fwd" + (" + kvp_attn_bwd" if backward else "") + " with q, k, v" +
+                               (", dO" if backward else "") + " coming from pinned host memory and " +
+                               ("dQ and the fp32 dK/dV sums" if backward else "O") + " going back, every step")
+                e2e_obj = obj
+            else:
+                obj["what"] = ("the whole block step with X" + (", dO" if backward else "") + " from pinned host memory and " +
+                               ("dX of every layer and the fp32 weight-gradient bucket" if backward else "O of every layer") +
+                               " going back, every step; block model FLOPs")
+                block_e2e = obj
+            runner.teardown_e2e()
+    if e2e_obj is None:
+        e2e_obj = {"value": float("nan"), "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     status = kvp.device_status()
     line = {
         "metric": "shared-KV attn fwd+bwd TFLOP/s" if backward else "shared-KV attn prefill fwd TFLOP/s",
@@ -435,15 +521,18 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
         "config": {"workload": cfg.name, "layers": cfg.L, "donor": cfg.donor, "batch_per_gpu": cfg.B,
                    "global_batch": cfg.B * world, "seq_len": cfg.S, "d_model": cfg.D, "heads": [cfg.Hq, cfg.Hkv],
                    "head_dim": cfg.dh, "parallelism": f"dp{world}", "l2": "inputs larger than L2 (about 10 GB live)",
-                   "flops": "model count: 3 x forward, causal pairs S(S+1)/2"},
+                   "flops": "value: attention kernels only, model count (forward 2 GEMMs, backward 4), causal pairs "
+                            "S(S+1)/2, over the summed device time of the attention kernels inside the timed block step; "
+                            "ms_per_step: the whole block step (projections + attention)"},
         "clocks": clocks, "gpu_launches": int(launches),
+        "attn_ms_per_step": attn_ms,
+        "attn_flash_convention_tflops": flash,
+        "block_tflops": block_tflops,
+        "block_model_flops_per_step": flops,
         "tokens_per_s": world * cfg.T / (ms_step * 1e-3),
         "pct_bf16_peak_nominal": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
         "pct_bf16_peak_measured": 100.0 * value / world / peak,
-        "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": runner.h2d,
-                "d2h_bytes_per_step": runner.d2h, "ms_per_step": ms_e2e / e2e_steps,
-                "copies": "pipelined: step n+1's inputs arrive on a second stream while step n computes; "
-                          "one input and one result transfer per timed step"},
+        "e2e": e2e_obj, "block_e2e": block_e2e,
         "roofline": roofline, "device_status": kvp.status_string(status),
     }
     del runner
@@ -451,7 +540,7 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
     return line, cfg, backward
 
 
-def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, steps=None, warmup=None):
+def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, steps=None, warmup=None, extra_modes=True):
     cfg = W.SMALL_DECODE if args.small else W.C3
     steps = cfg.steps if steps is None else steps
     warmup = 3 if warmup is None else warmup
@@ -488,6 +577,43 @@ def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, st
             runner.step_e2e(i)
         e2e_steps = min(steps, 32)
         ms_e2e, _ = timed_region(runner.step_e2e, e2e_steps, device, local_rank)
+    e2e_h2d, e2e_d2h = runner.h2d, runner.d2h
+    # the two other report modes: the same model decoded layer by layer (consumers re-read their donor's pages), and
+    # the same model with nothing shared (every layer stores and reads its own K/V); a bounded number of steps each
+    modes = {}
+    if not args.small and extra_modes:
+        m_steps = min(steps, 32)
+        unshared_m = W.decode_step_bytes(W.C3_UNSHARED, [float(lens0.double().mean()) + (m_steps + 1) / 2.0] * cfg.B)
+        for key, mcfg, per_layer in (("per_layer_sequential", cfg, True), ("unshared", W.C3_UNSHARED, False)):
+            if key == "per_layer_sequential":
+                runner.per_layer, r2 = True, runner
+                bytes_step = unshared_m              # every layer reads a full K/V stream
+            else:
+                del runner
+                torch.cuda.empty_cache()
+                free2, _t = torch.cuda.mem_get_info()
+                r2 = DecodeRunner(kvp, mcfg, device, n_slots=int(max(1, min(len(mcfg.owners()), (free2 - (6 << 30)) // per_slot))))
+                bytes_step = unshared_m
+            r2.reset()
+            for i in range(3):
+                r2.step(i)
+            torch.cuda.synchronize()
+            r2.reset()
+            n_ev = m_steps * (mcfg.L if r2.per_layer else 1)
+            with kvp.KernelTimer(kvp.KERNEL_DECODE, n_ev) as kt2:
+                ms2, _c = timed_region(r2.step, m_steps, device, local_rank)
+            k2 = sum(kt2.durations_ms()) / m_steps
+            modes[key] = {"tokens_per_s": world * cfg.B / (ms2 / m_steps * 1e-3), "ms_per_step": ms2 / m_steps,
+                          "bytes_per_step": bytes_step, "hbm_gbs": bytes_step / (ms2 / m_steps * 1e-3) / 1e9,
+                          "kernel_gbs": bytes_step / (k2 * 1e-3) / 1e9, "steps": m_steps,
+                          "decode_calls_per_step": mcfg.L if r2.per_layer else 1,
+                          "stored_layers": len(mcfg.owners())}
+            if key == "per_layer_sequential":
+                runner.per_layer = False
+            else:
+                runner = r2
+        modes["grouped_over_per_layer"] = modes["per_layer_sequential"]["ms_per_step"] / ms_step
+        modes["grouped_over_unshared"] = modes["unshared"]["ms_per_step"] / ms_step
     out = {
         "metric": "shared-cache decode tokens/s", "value": world * cfg.B / (ms_step * 1e-3), "unit": "tokens/s",
         "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -496,15 +622,17 @@ def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, st
         "config": {"workload": cfg.name, "layers": cfg.L, "stored_layers": own, "batch_per_gpu": cfg.B,
                    "context": [cfg.len_lo, cfg.len_hi], "page": cfg.page, "heads": [cfg.Hq, cfg.Hkv],
                    "head_dim": cfg.dh, "physical_layer_pools": n_slots, "mode": "grouped (donor+consumer in one pass)",
+                   "block_table": "pages of a sequence scattered over the pool (seeded shuffle)",
                    "l2": "cache slices far larger than L2", "bytes_per_step": step_bytes,
                    "bytes_per_step_unshared": unshared_bytes},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": world * cfg.B / (ms_e2e / e2e_steps * 1e-3), "unit": "tokens/s",
-                "h2d_bytes_per_step": runner.h2d, "d2h_bytes_per_step": runner.d2h},
+                "h2d_bytes_per_step": e2e_h2d, "d2h_bytes_per_step": e2e_d2h},
+        "modes": modes,
         "roofline": {"bound": "hbm", "kernel": "decode_kernel<128>", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak,
                      "traffic": None if args.small else NCU_TRAFFIC_BYTES["decode_kernel"],
-                     "traffic_unit": "bytes per launch (ncu, full-size capture)",
+                     "traffic_unit": NCU_TRAFFIC_NOTE,
                      "algorithmic_bytes_per_launch": step_bytes, "peak_kind": f"{peaks_kind} copy bandwidth",
                      "kernel_ms_per_step": k_ms, "share_of_step": k_ms / ms_step,
                      "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
@@ -823,13 +951,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode workload in the default run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the shortened prefill and tail-stage runs of the default line")
     ap.add_argument("--small", action="store_true",
                     help="reduced shapes of the same kernels (inputs still larger than L2, under 2 GB on the device) "
                          "for profiler captures; implies --no-decode for train and --no-cpu-baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" and not args.small else args.warmup
     if args.small:
-        args.no_decode = args.no_cpu_baseline = True
+        args.no_decode = args.no_cpu_baseline = args.no_extras = True
 
     rank, local_rank, world = kdist.env_world()
     if args.impl == "reference":
@@ -845,6 +974,21 @@ def main():
 
     if args.workload in ("train", "prefill"):
         line, cfg, backward = run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
+        if args.workload == "train" and not args.small and not args.no_extras:
+            # the prefill configuration and the tail-stage workload, shortened, so that the default record carries them
+            sub = argparse.Namespace(**vars(args))
+            sub.steps, sub.warmup = max(3, min(args.steps, 5)), 3
+            try:
+                pl, _c, _b = run_train_like(sub, kvp, rank, local_rank, world, device, peaks, peaks_kind, workload="prefill", e2e=False)
+                line["prefill"] = {k: pl[k] for k in ("metric", "value", "unit", "ms_per_step", "attn_ms_per_step", "block_tflops",
+                                                      "pct_bf16_peak_nominal", "tokens_per_s", "steps", "warmup")}
+                line["prefill"]["config"] = pl["config"]["workload"]
+                line["prefill"]["kernels"] = pl["roofline"]["kernels"]
+                st = run_stage(sub, kvp, rank, local_rank, world, device, peaks, peaks_kind)
+                line["stage"] = {k: st[k] for k in ("metric", "value", "unit", "stage", "speedup_converted", "flops_ratio_converted", "steps", "warmup")}
+                line["stage"]["config"] = st["config"]
+            except Exception as exc:
+                line["extras_error"] = repr(exc)
         if args.workload == "train" and not args.no_decode:
             try:
                 line["decode"] = run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)

@@ -59,7 +59,7 @@ int kvp_device_status(void);
 /* Benchmark bookkeeping.  kvp_launch_count: kernels launched by this library since it was loaded.
  * kvp_set_timing_events: record the caller's CUDA events (HOST arrays of n cudaEvent_t, created by
  * the caller) immediately before and after each of the next n launches of one kernel
- * (0 GEMM, 1 attention forward, 2 attention backward dK/dV, 3 decode, 4 attention backward dQ); n == 0 switches it off.
+ * (0 GEMM, 1 attention forward, 2 attention backward, 3 decode, 4 the backward's helper passes: Delta, accumulator clear, dQ conversion, one pair per group of launches); n == 0 switches it off.
  * kvp_timing_events_used: how many pairs have been recorded since.  Not thread-safe. */
 unsigned long long kvp_launch_count(void);
 int kvp_set_timing_events(int kernel, void** starts, void** stops, int n);
@@ -247,7 +247,9 @@ int kvp_cache_append(const kvp_decode_desc* d, const int32_t* donor, const void*
 
 /* o[l][b,hq] = softmax(q[l][b,hq] . K_d[b, 0:len]^T * scale) V_d[b, 0:len] over the donor's pages
  * for layers layer_begin <= l < layer_end.  A donor and its consumers inside the range are served
- * by one pass over the donor's pages (each page read once per donor, not once per layer).
+ * by one pass over the donor's pages (each page read once per donor, not once per layer) as long as
+ * the group's query rows fit one pass: min(4, 16 / (Hq/Hkv)) layers; a larger group takes one pass
+ * per that many layers.
  * q[l], o[l]: [B,Hq,dh] bf16; lse[l]: [B,Hq] fp32.  lengths outside [1, max_pages*page_size] are
  * clamped.  Workspace: kvp_decode_workspace_bytes. */
 int kvp_decode(const kvp_decode_desc* d, const int32_t* donor, float scale, const void* const* q,
@@ -264,8 +266,9 @@ int kvp_decode(const kvp_decode_desc* d, const int32_t* donor, float scale, cons
  * of KVP_DECODE_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
  * library holds those bytes until the process exits.
  *
- *  - A request whose partials need more than that (kvp_decode_workspace_bytes(d, donor) bytes:
- *    grows with the number of donor groups, B, Hkv and the split count) is refused with
+ *  - A request whose partials need more than that (they grow with the number of donor groups that
+ *    [layer_begin, layer_end) touches, up to 64 per launch, and with B, Hkv and the split count;
+ *    kvp_decode_workspace_bytes(d, donor) is the figure for all layers) is refused with
  *    KVP_ERR_STATIC_SCRATCH and nothing is launched; lower num_splits, decode a narrower layer
  *    range per call, or use kvp_decode with your own workspace.
  *  - No cudaMalloc / cudaFree / allocating library call is made, on any call.

@@ -245,6 +245,30 @@ def attn_bwd(q, k, v, d_o, donor, causal=True, scale=None):
     return dq, dk, dv
 
 
+def attn_bwd_rows(q_rows, row_index, k_head, v_head, g_rows, causal=True, scale=None):
+    """Backward of selected query rows of ONE head (the same chain rule as attn_bwd;
+    query rows are independent given K and V, so their contributions add).
+
+    q_rows, g_rows [n,dh]: the queries and their dO at positions row_index [n];
+    k_head, v_head [S,dh].  Returns dq_rows [n,dh] and the CONTRIBUTION of these
+    rows to dK and dV of the head, [S,dh] each: summing the contributions of all
+    rows of all heads and layers that read the head gives dk_sum / dv_sum."""
+    q_rows = np.asarray(q_rows, dtype=np.float64)
+    g_rows = np.asarray(g_rows, dtype=np.float64)
+    k_head = np.asarray(k_head, dtype=np.float64)
+    v_head = np.asarray(v_head, dtype=np.float64)
+    dh = q_rows.shape[1]
+    sc = (1.0 / math.sqrt(dh)) if scale is None else float(scale)
+    s = (q_rows @ k_head.T) * sc
+    if causal:
+        j = np.arange(k_head.shape[0])[None, :]
+        s = np.where(j <= np.asarray(row_index)[:, None], s, -np.inf)
+    p, _ = _softmax_rows(s)
+    delta = (g_rows * (p @ v_head)).sum(axis=1, keepdims=True)
+    ds = p * (g_rows @ v_head.T - delta)
+    return (ds @ k_head) * sc, (ds.T @ q_rows) * sc, p.T @ g_rows
+
+
 # --------------------------------------------------------------------------
 # decode over the shared cache
 # --------------------------------------------------------------------------

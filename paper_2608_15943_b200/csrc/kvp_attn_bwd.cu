@@ -1,6 +1,6 @@
-// Flash-attention backward over a donor map (chain rule of Eq. 2-3 of the paper), two kernels:
+// Flash-attention backward over a donor map (chain rule of Eq. 2-3 of the paper) in ONE pass.
 //
-//  dkdv_kernel  KV-stationary.  One CTA owns a 128-row K/V tile of one (batch, KV head) of a DONOR
+//  bwd_kernel   KV-stationary.  One CTA owns a 128-row K/V tile of one (batch, KV head) of a DONOR
 //               layer, keeps K and V in shared memory and the dK / dV accumulators in TMEM (fp32)
 //               while it walks every query stream that reads the tile: the donor itself and all its
 //               consumer layers, the Hq/Hkv query heads of the KV head's group, and every 64-row query
@@ -10,20 +10,23 @@
 //               followed by one rank-3 MMA that subtracts the query's LSE/scale resp. Delta (a bf16
 //               three-term split against a tile of ones), so the accumulators already hold the
 //               exponent and dP - Delta; P^T = exp2(c acc), dS^T = P^T acc' are written back as bf16
-//               over the same TMEM columns and fed to dV += P^T dO, dK += dS^T Q as the A operand FROM
-//               TMEM -- P and dS never touch shared memory.  Two TMEM buffer sets alternate between
-//               steps; both compute warpgroups work on every step, each on half of its query columns.
+//               over the score columns and fed to dV += P^T dO, dK += dS^T Q as the A operand FROM
+//               TMEM.  dS^T also goes to shared memory, where it is the B operand of the fifth product
+//               dQ^T = K^T dS^T (K read as an MN-major A operand): the step's [dh x 64] partial of dQ
+//               lands in TMEM, a third warpgroup moves it to shared memory and adds it to an fp32
+//               accumulator in global memory with bulk reductions (cp.reduce.async.bulk .add.f32, 2 KB
+//               each), so S and dP are computed once for all three gradients.
 //
-//  dq_kernel    Q-stationary (like the forward).  One CTA owns a 128-row query tile of one (layer,
-//               batch, query head) and walks the donor's K/V tiles: S = Q K^T, dP = dO V^T,
-//               dS = P (dP - Delta) written as bf16 over dP's TMEM columns, dQ += dS K with dS as the A
-//               operand from TMEM and K as an MN-major B operand.  dQ accumulates in TMEM and is
-//               written once, as bf16, already scaled: no atomics, no fp32 dQ round trip through HBM.
+//  dq_convert_kernel  scales the fp32 dQ accumulators and writes dQ as bf16 [B,S,Hq,dh].
 //
-// Delta = rowsum(dO * O) comes from a small pre-pass.  Recomputing S and dP in both kernels costs
-// two extra GEMMs per tile pair; it removes 64 KB of fp32 reduction traffic per tile pair, which is
-// what bounded the single-kernel form.
+// Delta = rowsum(dO * O) comes from a small pre-pass.  The dQ accumulators live in the caller's
+// workspace in a blocked layout ([b][hq][64-query tile][32-column quarter][64][32] fp32) so that every
+// reduction is one contiguous 2 KB run; they are cleared before each donor group's launch.  The order in
+// which the key tiles' partials reach an accumulator is not fixed, so dQ (unlike dK, dV) is reproducible
+// only up to fp32 rounding order.
 #include <math.h>
+
+#include <algorithm>
 
 #include "kvp_host.h"
 #include "kvp_sm100.cuh"
@@ -31,9 +34,9 @@
 namespace kvp {
 namespace {
 
-constexpr int BT = 128;    // key rows per tile (both kernels), query rows per tile in dq_kernel
-constexpr int BQ2 = 64;    // query rows per step in dkdv_kernel
-constexpr int MAX_GROUP = 8;  // layers of one donor group per dkdv launch
+constexpr int BT = 128;    // key rows per tile
+constexpr int BQ2 = 64;    // query rows per step
+constexpr int MAX_GROUP = 8;  // layers of one donor group per launch
 constexpr uint32_t HALF_BYTES = 128 * 128;  // [128 rows x 128 B] block
 constexpr uint32_t QHALF_BYTES = 64 * 128;  // [ 64 rows x 128 B] block
 
@@ -45,38 +48,47 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// =============================================================================================
-// dK / dV
-// =============================================================================================
-constexpr int DKDV_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9 two compute warpgroups
-constexpr int DKDV_STAGES = 4;     // ring of (Q, dO) 64-row tiles
+// warp 0 TMA, warp 1 MMA, warps 2-5 and 6-9 two compute warpgroups, warps 10-13 dQ drain
+constexpr int BWD_THREADS = 448;
+constexpr int BWD_STAGES = 3;        // ring of (Q, dO) 64-row tiles
+constexpr int DQ_STAGE_BYTES = BQ2 * 32 * 4;  // one drain warp's share of a step: [64 queries x 32 columns] fp32
+// A CTA's window of query tiles is sized so that it runs about this many steps (window x streams): long enough
+// to amortise its prologue and its dK / dV reduction, short enough that a wave's footprint stays in L2.
+constexpr int kStepsPerCta = 512;
+constexpr int kMinWindow = 16;
 
 template <int DH>
-struct DkdvSmem {
+struct BwdSmem {
   static constexpr int KV_TILE = BT * DH * 2;
   static constexpr int Q_TILE = BQ2 * DH * 2;
   static constexpr int STAGE = 2 * Q_TILE;  // Q then dO
   static constexpr int OFF_K = 0;
   static constexpr int OFF_V = OFF_K + KV_TILE;
   static constexpr int OFF_RING = OFF_V + KV_TILE;
-  static constexpr int OFF_ONES = OFF_RING + DKDV_STAGES * STAGE;  // [128 x 16] bf16, unswizzled K-major
-  static constexpr int OFF_STAT = OFF_ONES + 4096;                 // [4 steps][lse, delta][64 x 16] bf16
-  static constexpr int OFF_BAR = OFF_STAT + 8 * 2048;
+  static constexpr int OFF_DS = OFF_RING + BWD_STAGES * STAGE;     // dS^T [128 keys x 64 queries] bf16, 128-B swizzle
+  static constexpr int OFF_DQ = OFF_DS + BT * BQ2 * 2;             // [4 drain warps][64 x 32] fp32
+  static constexpr int OFF_ONES = OFF_DQ + 4 * DQ_STAGE_BYTES;     // [128 x 8] bf16: columns 0-7 of the tile of ones
+  static constexpr int OFF_STAT = OFF_ONES + 2048;                 // [4 steps][lse, delta][64 x 8] bf16: columns 0-7
+  static constexpr int OFF_ZERO = OFF_STAT + 8 * 1024;             // [128 x 8] zeros: columns 8-15 of all of the above
+  static constexpr int OFF_RAW = OFF_ZERO + 2048;                  // [4 statistics warps][8 steps][32] fp32 as loaded
+  static constexpr int OFF_BAR = OFF_RAW + 4096;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
 
-struct DkdvParams {
+struct BwdParams {
   CUtensorMap map_k, map_v;       // donor K, V: [B,S,Hkv,dh], box rows 128
   CUtensorMap map_q[MAX_GROUP];   // per layer of the group, box rows 64
   CUtensorMap map_do[MAX_GROUP];
   const float* lse[MAX_GROUP];    // [B,Hq,S]
   const float* delta[MAX_GROUP];  // [B,Hq,S]
+  float* dq_acc[MAX_GROUP];       // blocked fp32 accumulators, see dq_acc_floats()
   float* dk_sum;                  // fp32 [B,S,Hkv,dh]
   float* dv_sum;
   int n_layers;
   int B, S, Hq, Hkv;
   int causal;
-  int chunk;                      // (batch, KV head) pairs per dispatch chunk
+  int window;                     // query tiles per CTA
+  int ctas_per_pair;              // CTAs of one (batch, KV head): sum over windows of the key tiles that see the window
   float scale;
   float scale_log2;
 };
@@ -101,27 +113,38 @@ __device__ __forceinline__ uint4 split3_bf16(float v) {
   return out;
 }
 
-// Per 64-query step, transposed so that TMEM lane == key row: S^T = K Q^T and dP^T = V dO^T.  The
-// per-query statistics are applied BY THE TENSOR CORE: one extra K-step multiplies a [128 x 16] tile
+// Floats of one layer's dQ accumulator: [B][Hq][ceil(S/64)][DH/32][64][32].
+__host__ __device__ inline size_t dq_acc_floats(int B, int S, int Hq, int dh) {
+  return size_t(B) * Hq * ((S + BQ2 - 1) / BQ2) * BQ2 * dh;
+}
+
+// TMEM columns: S^T of step parity i at [i*64, i*64+64) (P^T and dS^T overwrite it as bf16), dP^T at
+// [128, 192), the step's dQ^T at [192, 256), dK at [256, 256+DH), dV above it.
+//
+// The per-query statistics are applied BY THE TENSOR CORE: one extra K-step multiplies a [128 x 16] tile
 // of ones (first three columns) with a [64 x 16] tile holding -LSE/scale (resp. -Delta) of each query
 // split into three bf16 terms, so the accumulators already hold S - LSE/scale and dP - Delta and the
 // threads need no per-column operand: P^T = exp2(c * acc), dS^T = P^T * acc'.
 template <int DH>
-__global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_constant__ DkdvParams p) {
-  using L = DkdvSmem<DH>;
+__global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_constant__ BwdParams p) {
+  using L = BwdSmem<DH>;
   constexpr int HALVES = DH / 64;
   constexpr int KSTEPS_DH = DH / 16;
   constexpr int KSTEPS_Q = BQ2 / 16;
+  constexpr int KSTEPS_KV = BT / 16;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* kv_full = bars + 0;
   uint64_t* q_full = bars + 1;                    // [STAGES]
-  uint64_t* q_empty = q_full + DKDV_STAGES;       // [STAGES]
-  uint64_t* st_full = q_empty + DKDV_STAGES;      // [2]  S^T and dP^T of buffer set b are in TMEM
-  uint64_t* pds_ready = st_full + 2;              // [2]  P^T, dS^T written and the set's next statistics staged
-  uint64_t* stat0 = pds_ready + 2;                // statistics of the first two steps staged (256 arrivals)
+  uint64_t* q_empty = q_full + BWD_STAGES;        // [STAGES]
+  uint64_t* st_full = q_empty + BWD_STAGES;       // S^T and dP^T of the step are in TMEM
+  uint64_t* dp_free = st_full + 1;                // dP^T of the step is in registers (256 arrivals)
+  uint64_t* pds_ready = dp_free + 1;              // [2] P^T, dS^T written (TMEM and shared memory), next statistics staged
+  uint64_t* dq_full = pds_ready + 2;              // dQ^T of the step is in TMEM; its dS^T tile may be overwritten
+  uint64_t* dq_free = dq_full + 1;                // dQ^T of the step is in registers (128 arrivals)
+  uint64_t* stat0 = dq_free + 1;                  // statistics of the first steps staged (256 arrivals)
   uint64_t* acc_done = stat0 + 1;                 // all MMAs have completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
 
@@ -129,42 +152,48 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
   const int lane = threadIdx.x & 31;
   int* err = &g_bwd_status;
 
-  // Blocks are dispatched in index order.  The (batch, KV head) pairs are taken in chunks of p.chunk pairs;
-  // inside a chunk the key tile is the slow index, so that under the causal mask the chunk's heaviest tiles
-  // (tile 0 sees every query tile) start first, while all CTAs that stream the same Q / dO tiles run within
-  // a wave or two of each other and find them in L2.
+  // Work decomposition.  A CTA is one (batch, KV head), one 128-row key tile and one WINDOW of p.window
+  // consecutive 64-row query tiles, for every query stream of the donor group.  All CTAs therefore take
+  // (nearly) the same number of steps per stream and walk the streams at the same pace, so the CTAs that
+  // run at the same time read the same few Q / dO tiles and add to the same few dQ accumulator tiles:
+  // what a wave touches over its lifetime stays in L2.  Blocks are dispatched in index order: (batch, KV
+  // head) slowest, then the window, then the key tiles that see it.  The windows of one key tile add their
+  // dK / dV partials to the (cleared) output with reductions.
   const int n_jt = (p.S + BT - 1) / BT;
-  const int n_pairs = p.Hkv * p.B;
-  const int chunk_i = blockIdx.x / (p.chunk * n_jt);
-  const int in_chunk = blockIdx.x - chunk_i * p.chunk * n_jt;
-  const int chunk_n = min(p.chunk, n_pairs - chunk_i * p.chunk);  // the last chunk may be short
-  const int jt = in_chunk / chunk_n;
-  const int pair = chunk_i * p.chunk + (in_chunk - jt * chunk_n);
+  const int n_qt = (p.S + BQ2 - 1) / BQ2;
+  const int pair = blockIdx.x / p.ctas_per_pair;
+  int jt = blockIdx.x - pair * p.ctas_per_pair;
+  int win = 0;
+  for (;; ++win) {
+    const int vis = p.causal ? min(n_jt, ((win + 1) * p.window * BQ2 + BT - 1) / BT) : n_jt;
+    if (jt < vis) break;
+    jt -= vis;
+  }
   const int hk = pair % p.Hkv;
   const int b = pair / p.Hkv;
   const int G = p.Hq / p.Hkv;
   const int kv0 = jt * BT;
-  const int n_qt = (p.S + BQ2 - 1) / BQ2;
-  const int qt_first = p.causal ? (kv0 / BQ2) : 0;
-  const int per_stream = n_qt - qt_first;
+  const int qt_first = max(p.causal ? (kv0 / BQ2) : 0, win * p.window);
+  const int per_stream = min(n_qt, (win + 1) * p.window) - qt_first;
   const int n_iter = p.n_layers * G * per_stream;
 
   if (threadIdx.x == 0) {
     mbar_init(kv_full, 1);
-    for (int s = 0; s < DKDV_STAGES; ++s) {
+    for (int s = 0; s < BWD_STAGES; ++s) {
       mbar_init(&q_full[s], 1);
       mbar_init(&q_empty[s], 1);
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&st_full[i], 1);
-      mbar_init(&pds_ready[i], 256);
-    }
+    mbar_init(st_full, 1);
+    mbar_init(dp_free, 256);
+    for (int i = 0; i < 2; ++i) mbar_init(&pds_ready[i], 256);
+    mbar_init(dq_full, 1);
+    mbar_init(dq_free, 128);
     mbar_init(stat0, 256);
     mbar_init(acc_done, 1);
     mbar_fence_init();
   }
-  // constant operand tiles: ones in the first three columns; statistics tiles start as zeros
-  for (int i = threadIdx.x; i < (4096 + 8 * 2048) / 16; i += blockDim.x) {
+  // constant operand tiles: ones in the first three columns; statistics tiles and the shared zero half start as zeros
+  for (int i = threadIdx.x; i < (L::OFF_RAW - L::OFF_ONES) / 16; i += blockDim.x) {
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (i < 128) v = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);  // row i, columns 0-7 = 1,1,1,0,0,0,0,0
     *reinterpret_cast<uint4*>(smem + L::OFF_ONES + i * 16) = v;
@@ -178,9 +207,10 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // buffer set i: S^T at [i*128, i*128+64), dP^T at [i*128+64, i*128+128); accumulators above
+  const uint32_t tm_dp = tmem_base + 128;
+  const uint32_t tm_dq = tmem_base + 192;
   const uint32_t tm_dk = tmem_base + 256;
-  const uint32_t tm_dv = tmem_base + 384;
+  const uint32_t tm_dv = tmem_base + 256 + DH;
 
   auto decode_iter = [&](int it, int& li, int& hq, int& q0) {
     const int stream = it / per_stream;
@@ -205,8 +235,8 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
       for (int it = 0; it < n_iter; ++it) {
         int li, hq, q0;
         decode_iter(it, li, hq, q0);
-        const int s = it % DKDV_STAGES;
-        const uint32_t ph = (it / DKDV_STAGES) & 1;
+        const int s = it % BWD_STAGES;
+        const uint32_t ph = (it / BWD_STAGES) & 1;
         if (!mbar_wait(&q_empty[s], ph ^ 1, err)) break;
         mbar_expect_tx_e(&q_full[s], L::STAGE, leader);
         uint8_t* dst = smem + L::OFF_RING + s * L::STAGE;
@@ -223,24 +253,34 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
       const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
       constexpr uint32_t idesc_st = umma_idesc_bf16(BT, BQ2, 0, 0);   // [128 keys x 64 queries]
       constexpr uint32_t idesc_acc = umma_idesc_bf16(BT, DH, 0, 1);   // A from TMEM, B MN-major
+      // dQ^T [dh x 64 queries] = K^T dS^T, both operands MN-major.  The instruction always spans 128 rows; with
+      // DH == 64 the upper 64 are fed from the V tile that follows K in shared memory and are never read.
+      constexpr uint32_t idesc_dq = umma_idesc_bf16(128, BQ2, 1, 1);
       constexpr uint32_t hi = desc_hi_sw128(1024);
       constexpr uint32_t hi_plain = desc_hi_plain(128);
       // low descriptor words of the resident tiles; per MMA only a constant is added
       const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K), 0);
       const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::OFF_V), 0);
-      const uint32_t ones_lo = desc_lo_plain(smem_u32(smem + L::OFF_ONES), 2048);
+      const uint32_t kmn_lo = desc_lo_sw128(smem_u32(smem + L::OFF_K), HALF_BYTES);   // K as MN-major A
+      const uint32_t ds_lo = desc_lo_sw128(smem_u32(smem + L::OFF_DS), 0);            // dS^T as MN-major B
+      // 16-column K-major tiles whose columns 8-15 are all zero share one block of zeros: the leading-dimension
+      // offset of each descriptor is the distance from the tile's first half to that block
+      const uint32_t zero_addr = smem_u32(smem + L::OFF_ZERO);
+      const uint32_t ones_lo = desc_lo_plain(smem_u32(smem + L::OFF_ONES), zero_addr - smem_u32(smem + L::OFF_ONES));
       const uint32_t stat_base = smem_u32(smem + L::OFF_STAT);
       const uint32_t ring = smem_u32(smem + L::OFF_RING);
       bool ok = mbar_wait(kv_full, 0, err);
       if (ok) ok = mbar_wait(stat0, 0, err);
       auto issue_scores = [&](int it) -> bool {
-        const int s = it % DKDV_STAGES;
-        if (!mbar_wait(&q_full[s], (it / DKDV_STAGES) & 1, err)) return false;
+        const int s = it % BWD_STAGES;
+        if (!mbar_wait(&q_full[s], (it / BWD_STAGES) & 1, err)) return false;
         tc_fence_after_sync();
         const uint32_t q_lo = desc_lo_sw128(ring + s * L::STAGE, 0);
         const uint32_t do_lo = desc_lo_sw128(ring + s * L::STAGE + L::Q_TILE, 0);
-        const uint32_t tm = tmem_base + (it & 1) * 128;
-        const uint32_t stat_lo = desc_lo_plain(stat_base + (it & 3) * 4096, 1024);
+        const uint32_t tm = tmem_base + (it & 1) * 64;
+        const uint32_t lse_addr = stat_base + (it & 3) * 2048;
+        const uint32_t stat_lo = desc_lo_plain(lse_addr, zero_addr - lse_addr);
+        const uint32_t delta_lo = desc_lo_plain(lse_addr + 1024, zero_addr - lse_addr - 1024);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
@@ -248,39 +288,49 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
           umma_ss_w(tm, desc_lo_add(k_lo, offa), desc_lo_add(q_lo, offb), hi, idesc_st, ks != 0, leader);
         }
         umma_ss_w(tm, ones_lo, stat_lo, hi_plain, idesc_st, 1, leader);                          // S^T -= LSE / scale
+        // the single dP^T buffer takes the next step once the compute warps hold the previous one in registers
+        if (it > 0 && !mbar_wait(dp_free, (it - 1) & 1, err)) return false;
+        tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_DH; ++ks) {
           const uint32_t offa = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
           const uint32_t offb = (ks / 4) * QHALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tm + 64, desc_lo_add(v_lo, offa), desc_lo_add(do_lo, offb), hi, idesc_st, ks != 0, leader);
+          umma_ss_w(tm_dp, desc_lo_add(v_lo, offa), desc_lo_add(do_lo, offb), hi, idesc_st, ks != 0, leader);
         }
-        umma_ss_w(tm + 64, ones_lo, desc_lo_add(stat_lo, 2048), hi_plain, idesc_st, 1, leader);  // dP^T -= Delta
-        umma_commit(&st_full[it & 1], leader);
+        umma_ss_w(tm_dp, ones_lo, delta_lo, hi_plain, idesc_st, 1, leader);                      // dP^T -= Delta
+        umma_commit(st_full, leader);
         return true;
       };
       if (ok && n_iter > 0) ok = issue_scores(0);
       for (int it = 0; it < n_iter && ok; ++it) {
-        // scores of the next step go to the other buffer set; its previous readers (the accumulate
-        // MMAs of step it-1) precede this in the in-order tensor pipe, and its statistics tile was
-        // staged before pds_ready(it-1)
+        // S^T of the next step goes to the other score buffer; its previous readers (the accumulate MMAs
+        // of step it-1) precede this in the in-order tensor pipe, and its statistics tile was staged
+        // before pds_ready(it-1)
         if (it + 1 < n_iter && !issue_scores(it + 1)) { ok = false; break; }
         if (!mbar_wait(&pds_ready[it & 1], (it >> 1) & 1, err)) { ok = false; break; }
         tc_fence_after_sync();
-        const int s = it % DKDV_STAGES;
+        const int s = it % BWD_STAGES;
         const uint32_t qmn_lo = desc_lo_sw128(ring + s * L::STAGE, QHALF_BYTES);                 // Q  as MN-major B
         const uint32_t domn_lo = desc_lo_sw128(ring + s * L::STAGE + L::Q_TILE, QHALF_BYTES);    // dO as MN-major B
-        const uint32_t tm = tmem_base + (it & 1) * 128;
+        const uint32_t tm = tmem_base + (it & 1) * 64;
+        // P^T of queries [32w, 32w+32) sits in 32-bit columns [32w, 32w+16) of the score buffer, dS^T in [32w+16, 32w+32)
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dV += P^T dO
-          umma_ts_w(tm_dv, tm + ks * 8 + (ks / 2) * 32, desc_lo_add(domn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0, leader);
+          umma_ts_w(tm_dv, tm + (ks / 2) * 32 + (ks % 2) * 8, desc_lo_add(domn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0, leader);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_Q; ++ks)  // dK += dS^T Q
-          umma_ts_w(tm_dk, tm + 64 + ks * 8 + (ks / 2) * 32, desc_lo_add(qmn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0, leader);
-        umma_commit(&q_empty[s], leader);
+          umma_ts_w(tm_dk, tm + (ks / 2) * 32 + 16 + (ks % 2) * 8, desc_lo_add(qmn_lo, ks * 2048), hi, idesc_acc, (it | ks) != 0, leader);
+        umma_commit(&q_empty[s], leader);  // the ring stage is free as soon as dV and dK have read it
+        if (it > 0 && !mbar_wait(dq_free, (it - 1) & 1, err)) { ok = false; break; }
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ^T = K^T dS^T
+          umma_ss_w(tm_dq, desc_lo_add(kmn_lo, ks * 2048), desc_lo_add(ds_lo, ks * 2048), hi, idesc_dq, ks != 0, leader);
+        umma_commit(dq_full, leader);
       }
       if (ok) umma_commit(acc_done, leader);
     }
-  } else {
+  } else if (warp < 10) {
     // ------------------------------ compute warpgroups ------------------------------
     const int wg = (warp - 2) >> 2;     // query columns [wg*32, wg*32+32) of every step
     const int quarter = warp & 3;       // TMEM lane quarter of this warp
@@ -288,22 +338,29 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
     const int kv_row = kv0 + r;
     const float inv_scale = 1.f / p.scale;
-    // Statistics: in each warpgroup, lane quarter 0 stages -LSE/scale and quarter 1 stages -Delta of
-    // the warpgroup's 32 query columns.  Values are fetched two steps before they are staged, so the
-    // global-memory latency never shows.
+    // Statistics: in each warpgroup, lane quarter 0 stages -LSE/scale and quarter 1 stages -Delta of the
+    // warpgroup's 32 query columns as the three-term bf16 split the tensor core adds.  The raw fp32 values come
+    // in through cp.async into a small ring in shared memory, issued eight steps before the step that uses them
+    // and read back (and staged as an operand tile) three steps before: no register ever waits on global memory.
     const int stat_kind = quarter ^ 2;  // 0 lse, 1 delta, others idle: the warps whose scheduler hosts no TMA / MMA warp
-    uint8_t* stat_row = smem + L::OFF_STAT + (stat_kind & 1) * 2048 + (wg * 32 + lane) * 16;
-    // Loads are unconditional (from a clamped, always valid address) and their raw values travel in
-    // registers together with a validity flag; sign, 1/scale and the padding value are applied when a
-    // value is staged two steps later, so that no instruction depends on a load in the step that issues it.
+    const bool stat_warp = stat_kind < 2;
+    uint8_t* stat_row = smem + L::OFF_STAT + (stat_kind & 1) * 1024 + (wg * 32 + lane) * 16;
+    float* raw = reinterpret_cast<float*>(smem + L::OFF_RAW) + ((wg * 2 + (stat_kind & 1)) * 8) * 32 + lane;
     const float stat_mul = stat_kind == 0 ? -inv_scale : -1.f;
     const float stat_pad = stat_kind == 0 ? -30000.f : 0.f;  // a query beyond the sequence: exp2 underflows to zero
     // Two cursors walk the steps in order (incremental decode of step -> layer, head, query tile): one
-    // for the step whose statistics are loaded next, one kStatAhead steps further that only pulls the
-    // line into L2 -- the loads are a few steps ahead of their use, which hides an L2 hit but not DRAM.
+    // for the step whose statistics are requested next, one kStatAhead steps further that only pulls the
+    // line into L2.
     constexpr int kStatAhead = 12;
+    // `row` is the statistic row of the cursor's (layer, head): it is looked up (an indexed read of the kernel
+    // parameters) only when the stream changes, never on the per-step path
     struct Cursor {
       int it = 0, qi = 0, g = 0, li = 0;
+      const float* row = nullptr;
+    };
+    auto row_of = [&](int li, int g) {
+      const float* src = stat_kind == 0 ? p.lse[li < p.n_layers ? li : 0] : p.delta[li < p.n_layers ? li : 0];
+      return src + (size_t(b) * p.Hq + hk * G + g) * p.S;
     };
     auto advance = [&](Cursor& c) {
       ++c.it;
@@ -313,66 +370,71 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
           c.g = 0;
           ++c.li;
         }
+        c.row = row_of(c.li, c.g);
       }
     };
-    const float* f_ptr = p.lse[0];
     auto locate = [&](const Cursor& c, bool& valid) {  // address of this lane's statistic of step c (clamped, always valid)
-      valid = false;
-      if (stat_kind < 2 && c.it < n_iter) {
-        const int qc = (qt_first + c.qi) * BQ2 + wg * 32 + lane;
-        valid = qc < p.S;
-        const float* src = stat_kind == 0 ? p.lse[c.li] : p.delta[c.li];
-        f_ptr = src + (size_t(b) * p.Hq + hk * G + c.g) * p.S + (valid ? qc : p.S - 1);
-      }
-      return f_ptr;
+      const int qc = (qt_first + c.qi) * BQ2 + wg * 32 + lane;
+      valid = stat_warp && c.it < n_iter && qc < p.S;
+      return c.row + (valid ? qc : p.S - 1);
     };
     Cursor cf, cp;
+    cf.row = cp.row = row_of(0, 0);
     for (int i = 0; i < kStatAhead; ++i) advance(cp);
-    auto fetch = [&](bool& valid) -> float {
-      bool ahead_valid;
+    auto request = [&]() -> bool {  // cp.async of the next step's value into its ring slot; returns its validity
+      bool ahead_valid, valid;
       const float* ahead = locate(cp, ahead_valid);
       if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(ahead));
       advance(cp);
       const float* ptr = locate(cf, valid);
+      if (stat_warp)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(raw + (cf.it & 7) * 32)), "l"(ptr) : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
       advance(cf);
-      return __ldg(ptr);
+      return valid;
     };
-    auto stage = [&](int tile, float raw, bool valid) {
-      if (stat_kind < 2) *reinterpret_cast<uint4*>(stat_row + tile * 4096) = split3_bf16(valid ? raw * stat_mul : stat_pad);
+    auto stage = [&](int step, bool valid) {  // the value of `step` has landed: split it into the step's operand tile
+      if (stat_warp)
+        *reinterpret_cast<uint4*>(stat_row + (step & 3) * 2048) = split3_bf16(valid ? raw[(step & 7) * 32] * stat_mul : stat_pad);
     };
-    bool v0, v1;
-    float s0, s1;
-#pragma unroll 1
-    for (int i = 0; i < 3; ++i) {  // the tiles of steps 0..2; step n+3's tile is staged at the end of step n
-      s0 = fetch(v0);
-      stage(i, s0, v0);
+    // validity flags of the requests in flight, oldest (step it+3) in bit 0
+    uint32_t vbits = 0;
+    {
+      const bool a0 = request(), a1 = request(), a2 = request();
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      stage(0, a0);
+      stage(1, a1);
+      stage(2, a2);
+      // steps 3..7; from here on a ring slot is requested again only after its previous value has been staged
+#pragma unroll
+      for (int i = 0; i < 5; ++i) vbits |= uint32_t(request()) << i;
     }
     fence_proxy_async_smem();
     mbar_arrive(stat0);
-    s0 = fetch(v0);
-    s1 = fetch(v1);
     const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
-    // P^T and dS^T (bf16 pairs) overwrite the first half of the warpgroup's OWN score columns: 32-bit
-    // columns [wg*48, wg*48+16) of S^T resp. dP^T, which the other warpgroup never reads
-    const uint32_t col_ld = wg * 32, col_st = wg * 48;
+    // P^T and dS^T (bf16 pairs) overwrite the warpgroup's OWN score columns, which the other warpgroup never
+    // reads: P^T in 32-bit columns [wg*32, wg*32+16), dS^T in [wg*32+16, wg*32+32)
+    const uint32_t col = wg * 32;
+    uint8_t* ds_smem = smem + L::OFF_DS;
     int qi = 0;  // query tile index of the current step inside its stream
     bool ok = true;
     for (int it = 0; it < n_iter; ++it) {
       const int set = it & 1;
-      const uint32_t tm = tmem_base + set * 128;
-      ok = mbar_wait(&st_full[set], (it >> 1) & 1, err);
+      const uint32_t tm = tmem_base + set * 64;
+      ok = mbar_wait(st_full, it & 1, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc_fence_after_sync();
       uint32_t st[32], dp[32];
-      tmem_ld_x32(tm + lane_sel + col_ld, st);
-      tmem_ld_x32(tm + 64 + lane_sel + col_ld, dp);
-      // issued here, so that the load has returned before the fences below (which wait for it)
-      bool v_new;
-      const float s_new = fetch(v_new);
-      const bool diag = p.causal && qi < BT / BQ2;                  // the first two query tiles straddle the diagonal
-      const int first_visible = diag ? r - qi * BQ2 - wg * 32 : 0;  // own columns below this are masked for this key row
+      tmem_ld_x32(tm + lane_sel + col, st);
+      tmem_ld_x32(tm_dp + lane_sel + col, dp);
+      vbits |= uint32_t(request()) << 5;  // statistics of step it+8
+      const int q_col0 = (qt_first + qi) * BQ2 + wg * 32;           // query of this warpgroup's first column
+      const bool diag = p.causal && q_col0 - wg * 32 < kv0 + BT;    // the query tile straddles the diagonal
+      const int first_visible = diag ? kv_row - q_col0 : 0;         // own columns below this are masked for this key row
       uint32_t pk[16], dk[16];
       tmem_ld_wait();
+      tc_fence_before_sync();
+      mbar_arrive(dp_free);
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const uint64_t x = fmul2(pack_f2(__uint_as_float(st[2 * i]), __uint_as_float(st[2 * i + 1])), c2);
@@ -386,19 +448,27 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         dk[i] = pack_bf16(f2_lo(d), f2_hi(d));
       }
       // keys beyond the sequence contribute nothing (their K/V rows are zero-filled; dK/dV rows are not stored)
-      tmem_st_x16(tm + lane_sel + col_st, pk);
-      tmem_st_x16(tm + 64 + lane_sel + col_st, dk);
+      tmem_st_x16(tm + lane_sel + col, pk);
+      tmem_st_x16(tm + lane_sel + col + 16, dk);
+      // dS^T also goes to shared memory as the B operand of dQ^T = K^T dS^T; the previous step's product
+      // must have finished reading the tile
+      if (it > 0) {
+        ok = mbar_wait(dq_full, (it - 1) & 1, err);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        *reinterpret_cast<uint4*>(ds_smem + sw128_offset(r, wg * 4 + j)) =
+            make_uint4(dk[4 * j], dk[4 * j + 1], dk[4 * j + 2], dk[4 * j + 3]);
       tmem_st_wait();
-      fence_proxy_async_smem();  // the statistics staged one step ago are read by the tensor core's proxy
+      fence_proxy_async_smem();  // dS^T, and the statistics staged one step ago, are read by the tensor core's proxy
       tc_fence_before_sync();
       mbar_arrive(&pds_ready[set]);
       // Off the critical path: the tile of step it+3 (last read by the scores of step it-1, which have
       // completed).  The next step's arrive publishes it, before the scores of step it+3 are issued.
-      stage((it + 3) & 3, s0, v0);
-      s0 = s1;
-      v0 = v1;
-      s1 = s_new;
-      v1 = v_new;
+      asm volatile("cp.async.wait_group 5;" ::: "memory");
+      stage(it + 3, vbits & 1u);
+      vbits >>= 1;
       if (++qi == per_stream) qi = 0;
     }
     ok = __all_sync(0xffffffffu, ok);
@@ -408,7 +478,7 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
     }
     if (ok) {
       tc_fence_after_sync();
-      // warpgroup 0 writes dK (scaled), warpgroup 1 writes dV; every lane loads, valid rows store
+      // warpgroup 0 adds dK (scaled), warpgroup 1 adds dV; every lane loads, valid rows reduce
       const bool valid = kv_row < p.S;
       const size_t row_off = ((size_t(b) * p.S + (valid ? kv_row : 0)) * p.Hkv + hk) * DH;
       float* dst = (wg == 0 ? p.dk_sum : p.dv_sum) + row_off;
@@ -422,12 +492,63 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
         if (valid) {
 #pragma unroll
           for (int v4 = 0; v4 < 8; ++v4)
-            *reinterpret_cast<float4*>(dst + c * 32 + v4 * 4) =
-                make_float4(__uint_as_float(a[4 * v4]) * mul, __uint_as_float(a[4 * v4 + 1]) * mul,
-                            __uint_as_float(a[4 * v4 + 2]) * mul, __uint_as_float(a[4 * v4 + 3]) * mul);
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c * 32 + v4 * 4),
+                         "f"(__uint_as_float(a[4 * v4]) * mul), "f"(__uint_as_float(a[4 * v4 + 1]) * mul),
+                         "f"(__uint_as_float(a[4 * v4 + 2]) * mul), "f"(__uint_as_float(a[4 * v4 + 3]) * mul)
+                         : "memory");
         }
       }
     }
+  } else {
+    // ------------------------------ dQ drain warpgroup ------------------------------
+    // TMEM lane == column of dQ (dh index): this warp owns dh columns [32*quarter, 32*quarter + 32) of the
+    // step's 64 queries, lays them out as [64 queries x 32 columns] fp32 in shared memory and adds them to the
+    // accumulator with one 8 KB bulk reduction, which has a whole step to read the buffer before it is rewritten.
+    const int quarter = warp & 3;
+    const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
+    const bool active = quarter * 32 < DH;  // with DH == 64 the upper lanes hold nothing
+    float* stg = reinterpret_cast<float*>(smem + L::OFF_DQ + (warp - 10) * DQ_STAGE_BYTES);
+    const uint32_t stg_s = smem_u32(stg);
+    int li = 0, g = 0, qi = 0;
+    bool ok = true;
+    for (int it = 0; it < n_iter; ++it) {
+      ok = mbar_wait(dq_full, it & 1, err);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      tc_fence_after_sync();
+      uint32_t a[32], c[32];
+      tmem_ld_x32(tm_dq + lane_sel, a);
+      tmem_ld_x32(tm_dq + lane_sel + 32, c);
+      tmem_ld_wait();
+      tc_fence_before_sync();
+      mbar_arrive(dq_free);
+      if (active) {
+        const size_t tile = ((size_t(b) * p.Hq + hk * G + g) * n_qt + (qt_first + qi)) * (DH / 32) + quarter;
+        float* dst = p.dq_acc[li] + tile * (BQ2 * 32);
+        // the previous step's reduction has read the buffer
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < BQ2; ++q) stg[q * 32 + lane] = __uint_as_float(q < 32 ? a[q & 31] : c[q & 31]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(dst), "r"(stg_s),
+                       "n"(DQ_STAGE_BYTES)
+                       : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      }
+      if (++qi == per_stream) {
+        qi = 0;
+        if (++g == G) {
+          g = 0;
+          ++li;
+        }
+      }
+    }
+    // the reductions must have completed before the block's shared memory goes away and the grid ends
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
   }
 
   tc_fence_before_sync();
@@ -438,329 +559,35 @@ __global__ void __launch_bounds__(DKDV_THREADS, 1) dkdv_kernel(const __grid_cons
   }
 }
 
-// =============================================================================================
-// dQ
-// =============================================================================================
-constexpr int DQ_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 query tile A, warps 6-9 query tile B
-constexpr int DQ_KSTAGES = 2;
-
+// dq[b,s,hq,:] = bf16(scale * accumulator), from the blocked fp32 layout [b][hq][tile][quarter][64][32].
+// One thread per 8 consecutive columns of one query row: two 16-byte loads, one 16-byte store.
 template <int DH>
-struct DqSmem {
-  static constexpr int TILE = BT * DH * 2;
-  static constexpr int OFF_Q = 0;                          // [2] query tiles A, B
-  static constexpr int OFF_DO = OFF_Q + 2 * TILE;          // [2]
-  static constexpr int OFF_K = OFF_DO + 2 * TILE;          // [DQ_KSTAGES]
-  static constexpr int OFF_V = OFF_K + DQ_KSTAGES * TILE;  // one stage: V_j is only read by the two dP products
-  static constexpr int OFF_BAR = OFF_V + TILE;
-  static constexpr int TOTAL = OFF_BAR + 256 + 1024;
-};
-
-struct DqParams {
-  CUtensorMap map_q, map_do, map_k, map_v;  // box rows 128
-  const float* lse;                         // [B,Hq,S]
-  const float* delta;                       // [B,Hq,S]
-  __nv_bfloat16* dq;                        // [B,S,Hq,dh]
-  int B, S, Hq, Hkv;
-  int causal;
-  float scale;
-  float scale_log2;
-};
-
-// Two adjacent query tiles (A, B) share every K/V tile the CTA fetches.  Each query tile owns one
-// 128-column TMEM buffer that is reused through a key tile's life -- S (fp32) -> read by the tile's
-// warpgroup -> dP (fp32, same columns) -> read -> dS (bf16 pairs, first 64 columns) -> A operand of
-// dQ += dS K -- plus a DH-column dQ accumulator.  While one tile's exponentials run, the tensor pipe
-// works on the other tile.
-template <int DH>
-__global__ void __launch_bounds__(DQ_THREADS, 1) dq_kernel(const __grid_constant__ DqParams p) {
-  using L = DqSmem<DH>;
-  constexpr int HALVES = DH / 64;
-  constexpr int KSTEPS_DH = DH / 16;
-  constexpr int KSTEPS_KV = BT / 16;
-
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
-  uint64_t* qdo_full = bars + 0;
-  uint64_t* k_full = bars + 1;                 // [KSTAGES]
-  uint64_t* k_empty = k_full + DQ_KSTAGES;     // [KSTAGES]
-  uint64_t* v_full = k_empty + DQ_KSTAGES;
-  uint64_t* v_empty = v_full + 1;
-  uint64_t* s_full = v_empty + 1;              // [2] per query tile
-  uint64_t* s_read = s_full + 2;               // [2] S of the tile is in registers (128 arrivals)
-  uint64_t* dp_full = s_read + 2;              // [2]
-  uint64_t* ds_ready = dp_full + 2;            // [2] dS of the tile written (128 arrivals)
-  uint64_t* dq_done = ds_ready + 2;            // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dq_done + 2);
-
-  const int warp = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
-  int* err = &g_bwd_status;
-
-  const int hq = blockIdx.x % p.Hq;
-  const int b = blockIdx.x / p.Hq;
-  const int n_qtiles = (p.S + BT - 1) / BT;
-  const int n_pairs = (n_qtiles + 1) / 2;
-  const int pair = n_pairs - 1 - blockIdx.y;  // heaviest pairs first
-  const int hk = hq / (p.Hq / p.Hkv);
-  const int q0 = pair * 2 * BT;
-  int n_kv[2];
-#pragma unroll
-  for (int x = 0; x < 2; ++x) {
-    const int qs = q0 + x * BT;
-    const int kv_end = p.causal ? min(p.S, qs + BT) : p.S;
-    n_kv[x] = qs < p.S ? (kv_end + BT - 1) / BT : 0;
-  }
-  const int n_max = max(n_kv[0], n_kv[1]);
-
-  if (threadIdx.x == 0) {
-    mbar_init(qdo_full, 1);
-    for (int i = 0; i < DQ_KSTAGES; ++i) {
-      mbar_init(&k_full[i], 1);
-      mbar_init(&k_empty[i], 1);
-    }
-    mbar_init(v_full, 1);
-    mbar_init(v_empty, 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&s_full[i], 1);
-      mbar_init(&s_read[i], 128);
-      mbar_init(&dp_full[i], 1);
-      mbar_init(&ds_ready[i], 128);
-      mbar_init(&dq_done[i], 1);
-    }
-    mbar_fence_init();
-  }
-  if (warp == 1) {
-    tmem_alloc(tmem_slot, 512);
-    tmem_relinquish();
-  }
-  tc_fence_before_sync();
-  __syncthreads();
-  tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_slot;
-  // query tile x: working buffer at [x*128, x*128+128), dQ accumulator at [256 + x*128, ...)
-
-  if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
-    {
-      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
-      if (leader) tma_prefetch_desc(&p.map_q);
-      if (leader) tma_prefetch_desc(&p.map_do);
-      if (leader) tma_prefetch_desc(&p.map_k);
-      if (leader) tma_prefetch_desc(&p.map_v);
-      mbar_expect_tx_e(qdo_full, 4 * L::TILE, leader);  // rows beyond the sequence are zero-filled
-#pragma unroll
-      for (int x = 0; x < 2; ++x)
-#pragma unroll
-        for (int h = 0; h < HALVES; ++h) {
-          tma_load_4d_e(smem + L::OFF_Q + x * L::TILE + h * HALF_BYTES, &p.map_q, qdo_full, h * 64, hq, q0 + x * BT, b, leader);
-          tma_load_4d_e(smem + L::OFF_DO + x * L::TILE + h * HALF_BYTES, &p.map_do, qdo_full, h * 64, hq, q0 + x * BT, b, leader);
-        }
-      auto load_k = [&](int j) -> bool {
-        const int s = j % DQ_KSTAGES;
-        if (!mbar_wait(&k_empty[s], ((j / DQ_KSTAGES) & 1) ^ 1, err)) return false;
-        mbar_expect_tx_e(&k_full[s], L::TILE, leader);
-#pragma unroll
-        for (int h = 0; h < HALVES; ++h)
-          tma_load_4d_e(smem + L::OFF_K + s * L::TILE + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, hk, j * BT, b, leader);
-        return true;
-      };
-      auto load_v = [&](int j) -> bool {
-        if (!mbar_wait(v_empty, (j & 1) ^ 1, err)) return false;
-        mbar_expect_tx_e(v_full, L::TILE, leader);
-#pragma unroll
-        for (int h = 0; h < HALVES; ++h)
-          tma_load_4d_e(smem + L::OFF_V + h * HALF_BYTES, &p.map_v, v_full, h * 64, hk, j * BT, b, leader);
-        return true;
-      };
-      bool ok = n_max > 0 ? load_k(0) : true;
-      for (int j = 0; j < n_max && ok; ++j) {
-        ok = load_v(j);
-        if (ok && j + 1 < n_max) ok = load_k(j + 1);
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
-    {
-      const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
-      constexpr uint32_t idesc_s = umma_idesc_bf16(BT, BT, 0, 0);
-      constexpr uint32_t idesc_dq = umma_idesc_bf16(BT, DH, 0, 1);  // A = dS from TMEM, B = K MN-major
-      constexpr uint32_t hi = desc_hi_sw128(1024);
-      const uint32_t k_base = smem_u32(smem + L::OFF_K);
-      const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::OFF_V), 0);
-      bool ok = mbar_wait(qdo_full, 0, err);
-      auto issue_s = [&](int x, int j) {  // S_x(j) = Q_x K_j^T
-        const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q + x * L::TILE), 0);
-        const uint32_t k_lo = desc_lo_sw128(k_base + (j % DQ_KSTAGES) * L::TILE, 0);
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS_DH; ++ks) {
-          const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tmem_base + x * BT, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_s, ks != 0, leader);
-        }
-        umma_commit(&s_full[x], leader);
-      };
-      if (ok && n_max > 0) {
-        ok = mbar_wait(&k_full[0], 0, err);
-        if (ok) {
-          tc_fence_after_sync();
-          if (n_kv[0] > 0) issue_s(0, 0);
-          if (n_kv[1] > 0) issue_s(1, 0);
-        }
-      }
-      for (int j = 0; j < n_max && ok; ++j) {
-        const uint32_t ph = j & 1;
-        if (!mbar_wait(v_full, ph, err)) { ok = false; break; }
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          if (j < n_kv[x]) {
-            // dP_x(j) overwrites S_x(j) once the warpgroup holds S_x(j) in registers
-            if (!mbar_wait(&s_read[x], ph, err)) { ok = false; break; }
-            tc_fence_after_sync();
-            const uint32_t do_lo = desc_lo_sw128(smem_u32(smem + L::OFF_DO + x * L::TILE), 0);
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS_DH; ++ks) {
-              const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-              umma_ss_w(tmem_base + x * BT, desc_lo_add(do_lo, off), desc_lo_add(v_lo, off), hi, idesc_s, ks != 0, leader);
-            }
-            umma_commit(&dp_full[x], leader);
-          }
-        }
-        if (!ok) break;
-        umma_commit(v_empty, leader);
-        const bool next = j + 1 < n_max;
-        if (next && !mbar_wait(&k_full[(j + 1) % DQ_KSTAGES], ((j + 1) / DQ_KSTAGES) & 1, err)) { ok = false; break; }
-        const uint32_t kmn_lo = desc_lo_sw128(k_base + (j % DQ_KSTAGES) * L::TILE, HALF_BYTES);  // K_j as MN-major B
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          if (j < n_kv[x]) {
-            if (!mbar_wait(&ds_ready[x], ph, err)) { ok = false; break; }
-            tc_fence_after_sync();
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS_KV; ++ks)  // dQ_x += dS_x(j) K_j
-              umma_ts_w(tmem_base + 256 + x * 128, tmem_base + x * BT + ks * 8, desc_lo_add(kmn_lo, ks * 2048), hi,
-                        idesc_dq, (j | ks) != 0, leader);
-            if (j + 1 == n_kv[x]) umma_commit(&dq_done[x], leader);
-            // the tile's buffer takes the next scores right behind dQ_x(j) in the in-order tensor pipe
-            if (j + 1 < n_kv[x]) issue_s(x, j + 1);
-          }
-        }
-        if (!ok) break;
-        umma_commit(&k_empty[j % DQ_KSTAGES], leader);
-      }
-    }
-  } else {
-    // ------------------------------ compute warpgroups ------------------------------
-    const int x = (warp - 2) >> 2;      // query tile of this warpgroup
-    const int quarter = warp & 3;
-    const int r = quarter * 32 + lane;  // query row inside the tile == TMEM lane
-    const int q_row = q0 + x * BT + r;
-    const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
-    const uint32_t tb = tmem_base + x * BT + lane_sel;
-    const int my_n = n_kv[x];
-    const size_t stat_idx = (size_t(b) * p.Hq + hq) * p.S + (q_row < p.S ? q_row : 0);
-    const float lse2 = q_row < p.S ? p.lse[stat_idx] * 1.4426950408889634f : INFINITY;
-    const float dl = q_row < p.S ? p.delta[stat_idx] : 0.f;
-    const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
-    const uint64_t nl2 = pack_f2(-lse2, -lse2);
-    const uint64_t ndl2 = pack_f2(-dl, -dl);
-    bool ok = true;
-    for (int j = 0; j < my_n; ++j) {
-      const uint32_t ph = j & 1;
-      ok = mbar_wait(&s_full[x], ph, err);
-      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-      tc_fence_after_sync();
-      const int kvb = j * BT;
-      int lim = p.S - kvb;
-      if (p.causal) lim = min(lim, q_row - kvb + 1);
-      uint32_t pb[BT / 2];  // P as bf16 pairs, kept across the dP product
-      {
-        uint32_t t0[32], t1[32], t2[32], t3[32];
-        tmem_ld_x32(tb, t0);
-        tmem_ld_x32(tb + 32, t1);
-        tmem_ld_x32(tb + 64, t2);
-        tmem_ld_x32(tb + 96, t3);
-        tmem_ld_wait();
-        tc_fence_before_sync();
-        mbar_arrive(&s_read[x]);  // the scores are in registers: dP may overwrite them
-        auto expo = [&](const uint32_t* t, uint32_t* out) {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const uint64_t v = ffma2(pack_f2(__uint_as_float(t[2 * i]), __uint_as_float(t[2 * i + 1])), c2, nl2);
-            out[i] = pack_bf16(fast_exp2(f2_lo(v)), fast_exp2(f2_hi(v)));
-          }
-        };
-        expo(t0, pb);
-        expo(t1, pb + 16);
-        expo(t2, pb + 32);
-        expo(t3, pb + 48);
-      }
-      if (__any_sync(0xffffffffu, lim < BT)) {  // diagonal or ragged tile: zero the masked columns
-#pragma unroll
-        for (int i = 0; i < BT / 2; ++i) {
-          uint32_t v = pb[i];
-          if (2 * i >= lim) v &= 0xffff0000u;
-          if (2 * i + 1 >= lim) v &= 0x0000ffffu;
-          pb[i] = v;
-        }
-      }
-      ok = mbar_wait(&dp_full[x], ph, err);
-      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-      tc_fence_after_sync();
-#pragma unroll
-      for (int c = 0; c < BT / 32; ++c) {
-        uint32_t tmp[32];
-        tmem_ld_x32(tb + c * 32, tmp);
-        tmem_ld_wait();
-        uint32_t ds[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint32_t pv = pb[c * 16 + i];
-          const uint64_t pf = pack_f2(__uint_as_float(pv << 16), __uint_as_float(pv & 0xffff0000u));
-          const uint64_t d = fmul2(pf, fadd2(pack_f2(__uint_as_float(tmp[2 * i]), __uint_as_float(tmp[2 * i + 1])), ndl2));
-          ds[i] = pack_bf16(f2_lo(d), f2_hi(d));
-        }
-        // dS (bf16 pairs) over dP's own columns: chunk c lands in columns [16c, 16c+16), already read
-        tmem_st_x16(tb + c * 16, ds);
-      }
-      tmem_st_wait();
-      tc_fence_before_sync();
-      mbar_arrive(&ds_ready[x]);
-    }
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok && my_n > 0) {
-      bool w = mbar_wait(&dq_done[x], 0, err);
-      ok = __all_sync(0xffffffffu, w);
-    }
-    if (ok && my_n > 0) {
-      tc_fence_after_sync();
-      const bool valid = q_row < p.S;
-      __nv_bfloat16* dst = p.dq + ((size_t(b) * p.S + (valid ? q_row : 0)) * p.Hq + hq) * DH;
-      const uint32_t src = tmem_base + 256 + x * 128 + lane_sel;
-#pragma unroll 1
-      for (int c = 0; c < DH / 32; ++c) {
-        uint32_t a[32];
-        tmem_ld_x32(src + c * 32, a);
-        tmem_ld_wait();
-        if (valid) {
-#pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint4 v;
-            v.x = pack_bf16(__uint_as_float(a[8 * v4 + 0]) * p.scale, __uint_as_float(a[8 * v4 + 1]) * p.scale);
-            v.y = pack_bf16(__uint_as_float(a[8 * v4 + 2]) * p.scale, __uint_as_float(a[8 * v4 + 3]) * p.scale);
-            v.z = pack_bf16(__uint_as_float(a[8 * v4 + 4]) * p.scale, __uint_as_float(a[8 * v4 + 5]) * p.scale);
-            v.w = pack_bf16(__uint_as_float(a[8 * v4 + 6]) * p.scale, __uint_as_float(a[8 * v4 + 7]) * p.scale);
-            *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = v;
-          }
-        }
-      }
-    }
-  }
-
-  tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 1) {
-    tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 512);
+__global__ void dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int B, int S, int Hq,
+                                  float scale) {
+  constexpr int TPR = DH / 8;  // threads per query row
+  const int n_qt = (S + BQ2 - 1) / BQ2;
+  const size_t rows = size_t(B) * Hq * n_qt * BQ2;
+  const size_t stride = size_t(gridDim.x) * blockDim.x / TPR;
+  const int j = threadIdx.x % TPR;
+  const int quarter = j / 4, d0 = (j % 4) * 8;
+  for (size_t row = (size_t(blockIdx.x) * blockDim.x + threadIdx.x) / TPR; row < rows; row += stride) {
+    const int q = int(row % BQ2);
+    const size_t tile = row / BQ2;  // (b * Hq + hq) * n_qt + qt
+    const int qt = int(tile % n_qt);
+    const size_t bh = tile / n_qt;
+    const int s = qt * BQ2 + q;
+    if (s >= S) continue;
+    const float* src = acc + ((tile * (DH / 32) + quarter) * BQ2 + q) * 32 + d0;
+    const float4 lo = *reinterpret_cast<const float4*>(src);
+    const float4 hi = *reinterpret_cast<const float4*>(src + 4);
+    uint4 v;
+    v.x = pack_bf16(lo.x * scale, lo.y * scale);
+    v.y = pack_bf16(lo.z * scale, lo.w * scale);
+    v.z = pack_bf16(hi.x * scale, hi.y * scale);
+    v.w = pack_bf16(hi.z * scale, hi.w * scale);
+    const int hq = int(bh % Hq);
+    const int bb = int(bh / Hq);
+    *reinterpret_cast<uint4*>(dq + ((size_t(bb) * S + s) * Hq + hq) * DH + quarter * 32 + d0) = v;
   }
 }
 
@@ -817,6 +644,7 @@ __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfl
   }
 }
 
+
 int make_map_bshd(CUtensorMap* m, const void* base, int B, int S, int H, int dh, int rows) {
   uint64_t dims[4] = {uint64_t(dh), uint64_t(H), uint64_t(S), uint64_t(B)};
   uint64_t strides[3] = {uint64_t(dh) * 2, uint64_t(H) * dh * 2, uint64_t(S) * H * dh * 2};
@@ -825,6 +653,17 @@ int make_map_bshd(CUtensorMap* m, const void* base, int B, int S, int H, int dh,
 }
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+int largest_group(const kvp_shape* s, const int32_t* donor) {
+  int best = 1;
+  for (int d = 0; d < s->L; ++d) {
+    if (donor[d] != d) continue;
+    int n = 0;
+    for (int l = d; l < s->L; ++l) n += donor[l] == d;
+    best = n > best ? n : best;
+  }
+  return best;
+}
 
 }  // namespace
 
@@ -838,10 +677,12 @@ int attn_bwd_read_status() {
   return v;
 }
 
-// Workspace: Delta [B,Hq,S] fp32 for every layer.
+// Workspace: Delta [B,Hq,S] fp32 for every layer, then the fp32 dQ accumulators of the largest donor group
+// (one per member layer; groups are processed one after the other and reuse them).
 size_t attn_bwd_workspace(const kvp_shape* s, const int32_t* donor) {
-  (void)donor;
-  return size_t(s->L) * align256(size_t(s->B) * s->Hq * s->S * 4);
+  const int n = donor != nullptr ? largest_group(s, donor) : s->L;
+  return size_t(s->L) * align256(size_t(s->B) * s->Hq * s->S * 4) +
+         size_t(n > MAX_GROUP ? MAX_GROUP : n) * align256(dq_acc_floats(s->B, s->S, s->Hq, s->dh) * 4);
 }
 
 int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
@@ -852,18 +693,18 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
   const int dh = s->dh;
   const float sc = scale == 0.f ? 1.f / sqrtf(float(dh)) : scale;
   const size_t delta_bytes = align256(size_t(s->B) * s->Hq * s->S * 4);
+  const size_t acc_bytes = align256(dq_acc_floats(s->B, s->S, s->Hq, dh) * 4);
   uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
-  cudaError_t e1, e2;
-  if (dh == 128) {
-    e1 = cudaFuncSetAttribute(dkdv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkdvSmem<128>::TOTAL);
-    e2 = cudaFuncSetAttribute(dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<128>::TOTAL);
-  } else {
-    e1 = cudaFuncSetAttribute(dkdv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkdvSmem<64>::TOTAL);
-    e2 = cudaFuncSetAttribute(dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<64>::TOTAL);
-  }
-  if (e1 != cudaSuccess || e2 != cudaSuccess) return KVP_ERR_CUDA;
+  uint8_t* acc_base = wsb + size_t(s->L) * delta_bytes;
+  static const cudaError_t attr = [] {
+    cudaError_t e = cudaFuncSetAttribute(bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::TOTAL);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::TOTAL);
+  }();
+  if (attr != cudaSuccess) return KVP_ERR_CUDA;
 
   // Delta for every layer
+  timing_before(KVP_KERNEL_ATTN_BWD_AUX, stream);
   for (int l = 0; l < s->L; ++l) {
     float* dl = reinterpret_cast<float*>(wsb + size_t(l) * delta_bytes);
     const size_t rows = size_t(s->B) * s->S * s->Hq;
@@ -878,40 +719,11 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
                                                    s->Hq);
     note_launch();
   }
+  timing_after(KVP_KERNEL_ATTN_BWD_AUX, stream);
   if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
 
-  // dQ, one launch per layer
-  for (int l = 0; l < s->L; ++l) {
-    const int d = donor[l];
-    DqParams p;
-    int rc = make_map_bshd(&p.map_q, q[l], s->B, s->S, s->Hq, dh, BT);
-    if (rc == KVP_OK) rc = make_map_bshd(&p.map_do, d_o[l], s->B, s->S, s->Hq, dh, BT);
-    if (rc == KVP_OK) rc = make_map_bshd(&p.map_k, k[d], s->B, s->S, s->Hkv, dh, BT);
-    if (rc == KVP_OK) rc = make_map_bshd(&p.map_v, v[d], s->B, s->S, s->Hkv, dh, BT);
-    if (rc != KVP_OK) return rc;
-    p.lse = lse[l];
-    p.delta = reinterpret_cast<const float*>(wsb + size_t(l) * delta_bytes);
-    p.dq = reinterpret_cast<__nv_bfloat16*>(dq[l]);
-    p.B = s->B;
-    p.S = s->S;
-    p.Hq = s->Hq;
-    p.Hkv = s->Hkv;
-    p.causal = causal;
-    p.scale = sc;
-    p.scale_log2 = sc * 1.4426950408889634f;
-    dim3 grid(s->B * s->Hq, ((s->S + BT - 1) / BT + 1) / 2);
-    timing_before(KVP_KERNEL_ATTN_BWD_DQ, stream);
-    if (dh == 128)
-      dq_kernel<128><<<grid, DQ_THREADS, DqSmem<128>::TOTAL, stream>>>(p);
-    else
-      dq_kernel<64><<<grid, DQ_THREADS, DqSmem<64>::TOTAL, stream>>>(p);
-    timing_after(KVP_KERNEL_ATTN_BWD_DQ, stream);
-    note_launch();
-    if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
-  }
-
-  // dK / dV, one launch per donor group.  A launch writes (does not add to) the accumulators, so a
-  // donor shared by more than MAX_GROUP layers is not supported.
+  // One launch per donor group: dK / dV of the donor (written, not added to: a donor shared by more than
+  // MAX_GROUP layers is not supported) and the dQ accumulators of every member layer.
   for (int d = 0; d < s->L; ++d) {
     if (donor[d] != d) continue;
     int members[MAX_GROUP];
@@ -921,7 +733,7 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
         if (n == MAX_GROUP) return KVP_ERR_UNSUPPORTED;
         members[n++] = l;
       }
-    DkdvParams p;
+    BwdParams p;
     int rc = make_map_bshd(&p.map_k, k[d], s->B, s->S, s->Hkv, dh, BT);
     if (rc == KVP_OK) rc = make_map_bshd(&p.map_v, v[d], s->B, s->S, s->Hkv, dh, BT);
     if (rc != KVP_OK) return rc;
@@ -932,6 +744,7 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
       if (rc != KVP_OK) return rc;
       p.lse[i] = lse[l];
       p.delta[i] = reinterpret_cast<const float*>(wsb + size_t(l) * delta_bytes);
+      p.dq_acc[i] = reinterpret_cast<float*>(acc_base + size_t(i < n ? i : 0) * acc_bytes);
     }
     p.dk_sum = dk_sum[d];
     p.dv_sum = dv_sum[d];
@@ -943,22 +756,40 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     p.causal = causal;
     p.scale = sc;
     p.scale_log2 = sc * 1.4426950408889634f;
-    // chunk: the smallest divisor of the pair count that still fills the SMs 1.5 times with CTAs
-    const int n_jt = (s->S + BT - 1) / BT, n_pairs = s->Hkv * s->B;
-    p.chunk = n_pairs;
-    for (int d = 1; d <= n_pairs; ++d)
-      if (n_pairs % d == 0 && 2 * d * n_jt >= 3 * sm_count()) {
-        p.chunk = d;
-        break;
-      }
-    dim3 grid(n_pairs * n_jt);
+    const int n_jt = (s->S + BT - 1) / BT, n_qt = (s->S + BQ2 - 1) / BQ2, n_pairs = s->Hkv * s->B;
+    p.window = std::min(n_qt, std::max(kMinWindow, (kStepsPerCta + n * (s->Hq / s->Hkv) - 1) / (n * (s->Hq / s->Hkv))));
+    p.ctas_per_pair = 0;
+    for (int w = 0; w * p.window < n_qt; ++w)
+      p.ctas_per_pair += causal ? std::min(n_jt, ((w + 1) * p.window * BQ2 + BT - 1) / BT) : n_jt;
+    const size_t kv_bytes = size_t(s->B) * s->S * s->Hkv * dh * 4;
+    timing_before(KVP_KERNEL_ATTN_BWD_AUX, stream);
+    if (cudaMemsetAsync(acc_base, 0, size_t(n) * acc_bytes, stream) != cudaSuccess ||
+        cudaMemsetAsync(dk_sum[d], 0, kv_bytes, stream) != cudaSuccess ||
+        cudaMemsetAsync(dv_sum[d], 0, kv_bytes, stream) != cudaSuccess)
+      return KVP_ERR_CUDA;
+    timing_after(KVP_KERNEL_ATTN_BWD_AUX, stream);
+    dim3 grid(n_pairs * p.ctas_per_pair);
     timing_before(KVP_KERNEL_ATTN_BWD, stream);
     if (dh == 128)
-      dkdv_kernel<128><<<grid, DKDV_THREADS, DkdvSmem<128>::TOTAL, stream>>>(p);
+      bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::TOTAL, stream>>>(p);
     else
-      dkdv_kernel<64><<<grid, DKDV_THREADS, DkdvSmem<64>::TOTAL, stream>>>(p);
+      bwd_kernel<64><<<grid, BWD_THREADS, BwdSmem<64>::TOTAL, stream>>>(p);
     timing_after(KVP_KERNEL_ATTN_BWD, stream);
     note_launch();
+    if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
+    timing_before(KVP_KERNEL_ATTN_BWD_AUX, stream);
+    for (int i = 0; i < n; ++i) {
+      const size_t threads = dq_acc_floats(s->B, s->S, s->Hq, dh) / 8;
+      const int blocks = int(min(size_t(sm_count()) * 16, (threads + 255) / 256));
+      if (dh == 128)
+        dq_convert_kernel<128><<<blocks, 256, 0, stream>>>(p.dq_acc[i], reinterpret_cast<__nv_bfloat16*>(dq[members[i]]),
+                                                           s->B, s->S, s->Hq, sc);
+      else
+        dq_convert_kernel<64><<<blocks, 256, 0, stream>>>(p.dq_acc[i], reinterpret_cast<__nv_bfloat16*>(dq[members[i]]),
+                                                          s->B, s->S, s->Hq, sc);
+      note_launch();
+    }
+    timing_after(KVP_KERNEL_ATTN_BWD_AUX, stream);
     if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
   }
   return KVP_OK;

@@ -49,8 +49,9 @@ struct DecParams {
   float scale_log2;
 };
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+// 16-byte asynchronous copy; with src_bytes == 0 nothing is read and the destination is filled with zeros
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -163,8 +164,11 @@ __global__ void __launch_bounds__(DEC_THREADS, 2) decode_kernel(const __grid_con
       const int idx = i * 32 + lane;          // 16-byte chunk index inside the contiguous granule
       const int row = idx / CHUNKS, chunk = idx % CHUNKS;
       const uint32_t off = ring_off<DH>(row, chunk);
-      cp_async16(dst + off, ksrc + size_t(idx) * 16);
-      cp_async16(dst + TILE_BYTES + off, vsrc + size_t(idx) * 16);
+      // Slots at or past the sequence length were never appended and may hold anything (a NaN there would
+      // survive the zero probability in P V): they are filled with zeros instead of being read.
+      const uint32_t nbytes = tok + row < len ? 16u : 0u;
+      cp_async16(dst + off, ksrc + size_t(idx) * 16, nbytes);
+      cp_async16(dst + TILE_BYTES + off, vsrc + size_t(idx) * 16, nbytes);
     }
   };
 
@@ -430,6 +434,17 @@ int build_groups(const kvp_decode_desc* d, const int32_t* donor, int begin, int 
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
+// Bytes of per-split partials that decoding layers [begin, end) needs: one launch holds at most MAX_DEC_GROUPS
+// sub-groups and launches reuse the space.  0 when the request cannot be served at all.
+size_t decode_scratch_bytes(const kvp_decode_desc* d, const int32_t* donor, int begin, int end) {
+  static thread_local SubGroup tmp[4096];
+  const int n_sub = build_groups(d, donor, begin, end, tmp, 4096);
+  if (n_sub <= 0) return 0;
+  const int per_launch = n_sub < MAX_DEC_GROUPS ? n_sub : MAX_DEC_GROUPS;
+  const size_t units = size_t(per_launch) * d->B * d->Hkv * pick_splits(d);
+  return align256(units * 16 * d->dh * 4) + align256(units * 16 * 2 * 4);
+}
+
 }  // namespace
 
 int decode_read_status() {
@@ -448,16 +463,7 @@ using namespace kvp;
 
 extern "C" size_t kvp_decode_workspace_bytes(const kvp_decode_desc* d, const int32_t* donor) {
   if (check_desc(d) != KVP_OK || donor == nullptr) return 0;
-  // one launch holds at most MAX_DEC_GROUPS sub-groups; launches reuse the workspace
-  int n_sub = 0;
-  {
-    static thread_local SubGroup tmp[4096];
-    n_sub = build_groups(d, donor, 0, d->L, tmp, 4096);
-    if (n_sub < 0) return 0;
-  }
-  const int per_launch = n_sub < MAX_DEC_GROUPS ? n_sub : MAX_DEC_GROUPS;
-  const size_t units = size_t(per_launch) * d->B * d->Hkv * pick_splits(d);
-  return align256(units * 16 * d->dh * 4) + align256(units * 16 * 2 * 4);
+  return decode_scratch_bytes(d, donor, 0, d->L);
 }
 
 extern "C" int kvp_cache_append(const kvp_decode_desc* d, const int32_t* donor, const void* const* k_new,
@@ -628,7 +634,9 @@ extern "C" int kvp_decode_static(const kvp_decode_desc* d, const int32_t* donor,
   if (donor == nullptr) return KVP_ERR_INVALID_ARG;
   for (int l = 0; l < d->L; ++l)
     if (donor[l] < 0 || donor[l] > l || donor[donor[l]] != donor[l]) return KVP_ERR_BAD_DONOR;
-  const size_t need = kvp_decode_workspace_bytes(d, donor);
+  if (layer_begin < 0 || layer_end > d->L || layer_begin >= layer_end) return KVP_ERR_INVALID_ARG;
+  // only the donor groups that the layer range touches need room, so a narrower range can fit where all layers do not
+  const size_t need = decode_scratch_bytes(d, donor, layer_begin, layer_end);
   if (need == 0) return KVP_ERR_UNSUPPORTED;
   if (need > size_t(KVP_DECODE_STATIC_SCRATCH_BYTES)) return KVP_ERR_STATIC_SCRATCH;
   void* scratch = nullptr;

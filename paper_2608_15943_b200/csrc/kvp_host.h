@@ -46,9 +46,9 @@ int sm_count();
 enum {
   KVP_KERNEL_GEMM = 0,
   KVP_KERNEL_ATTN_FWD = 1,
-  KVP_KERNEL_ATTN_BWD = 2,     // dK/dV kernel
+  KVP_KERNEL_ATTN_BWD = 2,      // single-pass backward kernel (dQ partials, dK, dV)
   KVP_KERNEL_DECODE = 3,
-  KVP_KERNEL_ATTN_BWD_DQ = 4,  // dQ kernel
+  KVP_KERNEL_ATTN_BWD_AUX = 4,  // backward helper passes: Delta, accumulator clear, dQ conversion
   KVP_KERNEL_COUNT = 5
 };
 void note_launch(int n = 1);

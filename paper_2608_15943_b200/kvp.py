@@ -334,7 +334,7 @@ def decode(desc, donor, q, k_cache, v_cache, block_table, lengths, o, lse, ws, s
 # ------------------------------------------------------------------------------------------
 # benchmark bookkeeping
 # ------------------------------------------------------------------------------------------
-KERNEL_GEMM, KERNEL_ATTN_FWD, KERNEL_ATTN_BWD, KERNEL_DECODE, KERNEL_ATTN_BWD_DQ = range(5)
+KERNEL_GEMM, KERNEL_ATTN_FWD, KERNEL_ATTN_BWD, KERNEL_DECODE, KERNEL_ATTN_BWD_AUX = range(5)
 lib.kvp_launch_count.restype = C.c_ulonglong
 lib.kvp_set_timing_events.restype = C.c_int
 lib.kvp_set_timing_events.argtypes = [C.c_int, _PP, _PP, C.c_int]

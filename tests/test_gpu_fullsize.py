@@ -18,13 +18,18 @@ def f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-def close(name, got, ref, rel=REL, abs_=ABS):
+def close(name, got, ref, rel=REL, abs_=ABS, sum_over_tokens=False):
+    """rel-L2 <= 1e-2 and max-abs <= 3e-2, literally, for bf16 outputs -- except where a value is so large that
+    bf16 storage alone cannot meet it (half an ulp of bf16 is 2^-8 |x| at worst, above 3e-2 from |x| = 7.7):
+    there the element's bound is that storage-rounding floor.  fp32 sums over many tokens (donor-group dK/dV
+    sums, weight gradients) take the max-abs bound relative to max(1, |ref|_inf)."""
     got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
     assert np.isfinite(got).all(), name
-    scale = max(1.0, float(np.abs(ref).max()))
     rl2 = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
     assert rl2 <= rel, f"{name}: rel-L2 {rl2:.3e}"
-    assert np.abs(got - ref).max() <= abs_ * scale, f"{name}: max-abs {np.abs(got - ref).max():.3e}"
+    bound = abs_ * max(1.0, float(np.abs(ref).max())) if sum_over_tokens else np.maximum(abs_, 2.0 ** -8 * np.abs(ref))
+    excess = np.abs(got - ref) - bound
+    assert excess.max() <= 0, f"{name}: max-abs {np.abs(got - ref).max():.3e}"
 
 
 def sample_rows(S, rng, n=10):
@@ -89,31 +94,17 @@ def test_c2_attention_forward_sampled_rows(c2_run):
         assert np.abs(f64(out["lse"][l][b, hq, rows]) - rl).max() <= LSE_TOL
 
 
-def _row_backward(q_rows, rows, kh, vh, g_rows, scale):
-    """Oracle arithmetic for single query rows: softmax row, Delta, dS row (chain rule of Eq. 2)."""
-    s = (q_rows @ kh.T) * scale
-    s = np.where(np.arange(kh.shape[0])[None, :] <= rows[:, None], s, -np.inf)
-    m = s.max(axis=1, keepdims=True)
-    p = np.exp(s - m)
-    p /= p.sum(axis=1, keepdims=True)
-    o = p @ vh
-    delta = (g_rows * o).sum(axis=1, keepdims=True)
-    ds = p * (g_rows @ vh.T - delta)
-    return p, ds
-
-
 def test_c2_attention_backward_sampled(c2_run):
     cfg, t, out = c2_run
     rng = np.random.default_rng(2)
     G = cfg.Hq // cfg.Hkv
-    scale = 1.0 / np.sqrt(cfg.dh)
     # dQ rows, one by one
     for (l, b, hq) in [(0, 0, 3), (4, 1, 20), (5, 1, 21), (7, 0, 31)]:
         d, hk = cfg.donor[l], hq // G
         rows = sample_rows(cfg.S, rng, 6)
         kh, vh = f64(out["k"][d][b, :, hk]), f64(out["v"][d][b, :, hk])
-        _, ds = _row_backward(f64(out["q"][l][b, rows, hq]), rows, kh, vh, f64(t["d_o"][l][b, rows, hq]), scale)
-        close(f"dq[{l},{b},{hq}]", f64(out["dq"][l][b, rows, hq]), (ds @ kh) * scale)
+        dq_rows, _dk, _dv = A.attn_bwd_rows(f64(out["q"][l][b, rows, hq]), rows, kh, vh, f64(t["d_o"][l][b, rows, hq]))
+        close(f"dq[{l},{b},{hq}]", f64(out["dq"][l][b, rows, hq]), dq_rows)
     # donor-group dK/dV of layer 4 for the last key rows of one (b, hk): only query rows >= j contribute,
     # summed over layers 4-7 and the four heads of the group (16 streams)
     b, hk, j0 = 1, 2, cfg.S - 300
@@ -125,11 +116,11 @@ def test_c2_attention_backward_sampled(c2_run):
         for h in range(G):
             hq = hk * G + h
             qr, gr = f64(out["q"][l][b, rows, hq]), f64(t["d_o"][l][b, rows, hq])
-            p, ds = _row_backward(qr, rows, kh, vh, gr, scale)
-            dk += (ds[:, j0:].T @ qr) * scale
-            dv += p[:, j0:].T @ gr
-    close("dk_sum[4] tail rows", f64(out["dk_sum"][4][b, j0:, hk]), dk)
-    close("dv_sum[4] tail rows", f64(out["dv_sum"][4][b, j0:, hk]), dv)
+            _dq, dk_c, dv_c = A.attn_bwd_rows(qr, rows, kh, vh, gr)
+            dk += dk_c[j0:]
+            dv += dv_c[j0:]
+    close("dk_sum[4] tail rows", f64(out["dk_sum"][4][b, j0:, hk]), dk, sum_over_tokens=True)
+    close("dv_sum[4] tail rows", f64(out["dv_sum"][4][b, j0:, hk]), dv, sum_over_tokens=True)
     # property at full size: rows of P sum to one, so sum_j dV[j] = sum over streams and rows of dO
     for d in (0, 4):
         members = [l for l in range(cfg.L) if cfg.donor[l] == d]
@@ -151,15 +142,15 @@ def test_c2_projection_backward_sampled(c2_run):
         x = f64(t["x"][l])
         dq = f64(out["dq"][l].reshape(cfg.T, nq))
         cols = [0, nq - 1] + [int(c) for c in rng.integers(0, nq, 3)]
-        close(f"dwq[{l}]", f64(out["dwq"][l][cols]), dq[:, cols].T @ x)
+        close(f"dwq[{l}]", f64(out["dwq"][l][cols]), dq[:, cols].T @ x, sum_over_tokens=True)
         toks = [0, cfg.T - 1] + [int(c) for c in rng.integers(0, cfg.T, 6)]
         dx = dq[toks] @ f64(t["wq"][l])
         if cfg.donor[l] == l:
             dk = A.round_bf16(f64(out["dk_sum"][l].reshape(cfg.T, -1)))
             dv = A.round_bf16(f64(out["dv_sum"][l].reshape(cfg.T, -1)))
             kc = [0, dk.shape[1] - 1, 517]
-            close(f"dwk[{l}]", f64(out["dwk"][l][kc]), dk[:, kc].T @ x)
-            close(f"dwv[{l}]", f64(out["dwv"][l][kc]), dv[:, kc].T @ x)
+            close(f"dwk[{l}]", f64(out["dwk"][l][kc]), dk[:, kc].T @ x, sum_over_tokens=True)
+            close(f"dwv[{l}]", f64(out["dwv"][l][kc]), dv[:, kc].T @ x, sum_over_tokens=True)
             dx = dx + dk[toks] @ f64(t["wk"][l]) + dv[toks] @ f64(t["wv"][l])
         close(f"dx[{l}]", f64(out["dx"][l][toks]), dx)
 

@@ -1,6 +1,9 @@
 """Parity of the CUDA path (through the C ABI) against the fp64 oracle, element by element, on the
-same seeded inputs.  Tolerances for bf16 outputs: rel-L2 <= 1e-2 and max-abs <= 3e-2 (scaled by
-max(1, |ref|_inf) for tensors whose entries exceed 1, i.e. sums over many tokens); LSE within 1e-3.
+same seeded inputs.  Tolerances: rel-L2 <= 1e-2 and max-abs <= 3e-2, literally, for every bf16 output
+(Q, K, V, O, dQ, dX, decode outputs) -- where a stored value exceeds 7.7 in magnitude the element's bound is
+bf16's own rounding floor 2^-8 |x| instead; LSE within 1e-3.  Only the fp32 SUMS over many tokens (the
+donor-group dK/dV sums, the weight gradients), whose entries grow with the number of summed terms,
+take the max-abs bound relative to max(1, |ref|_inf) -- the call sites say `sum_over_tokens=True`.
 Integer / index work (planner, donor map) is bit-exact and tested without a GPU."""
 import math
 
@@ -32,17 +35,19 @@ def f64l(ts):
     return [f64(t) for t in ts]
 
 
-def close(name, got, ref, rel=REL, abs_=ABS):
+def close(name, got, ref, rel=REL, abs_=ABS, sum_over_tokens=False):
     got = f64(got) if isinstance(got, torch.Tensor) else np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
     assert np.isfinite(got).all(), f"{name}: non-finite output"
     diff = np.abs(got - ref)
-    scale = max(1.0, float(np.abs(ref).max()))
     if np.linalg.norm(ref) > 1e-6 * math.sqrt(ref.size):   # an exactly-zero reference has no relative error
         rl2 = np.linalg.norm(got - ref) / np.linalg.norm(ref)
         assert rl2 <= rel, f"{name}: rel-L2 {rl2:.3e} > {rel}"
-    assert diff.max() <= abs_ * scale, f"{name}: max-abs {diff.max():.3e} > {abs_ * scale:.3e}"
+    # a bf16 value of magnitude above 7.7 cannot be stored to within 3e-2 (half an ulp is up to 2^-8 |x|):
+    # there the element's bound is that storage-rounding floor; below it the bound is the literal one
+    bound = abs_ * max(1.0, float(np.abs(ref).max())) if sum_over_tokens else np.maximum(abs_, 2.0 ** -8 * np.abs(ref))
+    assert (diff - bound).max() <= 0, f"{name}: max-abs {diff.max():.3e} > {abs_:.1e}"
 
 
 def lse_close(name, got, ref):
@@ -84,10 +89,10 @@ def test_gemm_all_layouts(kvp, M, N, K, a_mn, b_mn):
         return
     c32 = torch.full((M, N), float("nan"), device="cuda")
     kvp.gemm(sa, sb, c32, a_mn, b_mn)
-    close("gemm f32", c32, ref, rel=1e-5, abs_=1e-4)
+    close("gemm f32", c32, ref, rel=1e-5, abs_=1e-4, sum_over_tokens=True)     # tight bounds, relative to |C|_inf
     c16 = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
     kvp.gemm(sa, sb, c16, a_mn, b_mn)
-    close("gemm bf16", c16, A.round_bf16(ref), rel=1e-3, abs_=1e-2)
+    close("gemm bf16", c16, A.round_bf16(ref), rel=1e-3, abs_=1e-2, sum_over_tokens=True)
     assert kvp.device_status() == kvp.OK
 
 
@@ -120,18 +125,18 @@ def test_c0_block_per_op_and_composed(kvp):
     for l in range(cfg.L):
         close(f"dq[{l}]", out["dq"][l], dq[l])
     for l in own:
-        close(f"dk_sum[{l}]", out["dk_sum"][l], dk[l])
-        close(f"dv_sum[{l}]", out["dv_sum"][l], dv[l])
+        close(f"dk_sum[{l}]", out["dk_sum"][l], dk[l], sum_over_tokens=True)
+        close(f"dv_sum[{l}]", out["dv_sum"][l], dv[l], sum_over_tokens=True)
     dqs = f64l(out["dq"])
     dks = [A.round_bf16(f64(a)) if a is not None else None for a in out["dk_sum"]]
     dvs = [A.round_bf16(f64(a)) if a is not None else None for a in out["dv_sum"]]
     dwq, dwk, dwv, dx = A.proj_bwd(x, wq, wk, wv, dqs, dks, dvs, cfg.donor)
     for l in range(cfg.L):
-        close(f"dwq[{l}]", out["dwq"][l], dwq[l])
+        close(f"dwq[{l}]", out["dwq"][l], dwq[l], sum_over_tokens=True)
         close(f"dx[{l}]", out["dx"][l], dx[l])
     for l in own:
-        close(f"dwk[{l}]", out["dwk"][l], dwk[l])
-        close(f"dwv[{l}]", out["dwv"][l], dwv[l])
+        close(f"dwk[{l}]", out["dwk"][l], dwk[l], sum_over_tokens=True)
+        close(f"dwv[{l}]", out["dwv"][l], dwv[l], sum_over_tokens=True)
 
     # --- composed: oracle end to end with bf16 rounding where the interface stores bf16 ---
     r = A.round_bf16
@@ -147,13 +152,13 @@ def test_c0_block_per_op_and_composed(kvp):
         close(f"composed o[{l}]", out["o"][l], oc[l])
         assert np.abs(f64(out["lse"][l]) - lsec[l]).max() <= 5e-3
         close(f"composed dq[{l}]", out["dq"][l], dqc[l])
-        close(f"composed dwq[{l}]", out["dwq"][l], dwqc[l])
+        close(f"composed dwq[{l}]", out["dwq"][l], dwqc[l], sum_over_tokens=True)
         close(f"composed dx[{l}]", out["dx"][l], dxc[l])
     for l in own:
-        close(f"composed dk_sum[{l}]", out["dk_sum"][l], dkc[l])
-        close(f"composed dv_sum[{l}]", out["dv_sum"][l], dvc[l])
-        close(f"composed dwk[{l}]", out["dwk"][l], dwkc[l])
-        close(f"composed dwv[{l}]", out["dwv"][l], dwvc[l])
+        close(f"composed dk_sum[{l}]", out["dk_sum"][l], dkc[l], sum_over_tokens=True)
+        close(f"composed dv_sum[{l}]", out["dv_sum"][l], dvc[l], sum_over_tokens=True)
+        close(f"composed dwk[{l}]", out["dwk"][l], dwkc[l], sum_over_tokens=True)
+        close(f"composed dwv[{l}]", out["dwv"][l], dwvc[l], sum_over_tokens=True)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -212,8 +217,8 @@ def test_attention_forward_and_backward_shapes(kvp, B, S, Hq, Hkv, dh, donor, ca
     for l in range(L):
         close(f"dq[{l}]", dq[l], rdq[l])
         if donor[l] == l:
-            close(f"dk_sum[{l}]", dk[l], rdk[l])
-            close(f"dv_sum[{l}]", dv[l], rdv[l])
+            close(f"dk_sum[{l}]", dk[l], rdk[l], sum_over_tokens=True)
+            close(f"dv_sum[{l}]", dv[l], rdv[l], sum_over_tokens=True)
     # too small a workspace is refused, not overrun
     if ws.numel() > 256:
         with pytest.raises(kvp.KvpError) as e:
@@ -327,6 +332,39 @@ def test_decode_against_oracle(kvp, L, donor, B, Hq, Hkv, dh, page, lens, ns):
     assert kvp.device_status() == kvp.OK
 
 
+def test_decode_ignores_never_appended_slots_even_if_they_hold_nan(kvp):
+    """Cache slots at or past lengths[b] were never appended (a pool from an uninitialised allocation, a
+    recycled page): whatever bit pattern they hold, NaN included, must not reach the output.  Every slot past
+    the length, in the straddling 16-token granule, the rest of its page and the unused pages, is set to NaN."""
+    L, donor, B, Hq, Hkv, dh, page = 2, [0, 0], 3, 8, 2, 128, 64
+    lens = [1, 70, 200]          # inside the first granule, straddling a granule, straddling a page
+    max_pages = 5
+    n_pages = B * max_pages
+    g = torch.Generator().manual_seed(11)
+    bt = torch.randperm(n_pages, generator=g).int().reshape(B, max_pages).cuda()
+    lengths = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    kc = [synth.normal((n_pages, Hkv, page, dh), 17, synth.tid(7, 0), 1.0, "cuda"), None]
+    vc = [synth.normal((n_pages, Hkv, page, dh), 17, synth.tid(8, 0), 1.0, "cuda"), None]
+    q = [synth.normal((B, Hq, dh), 17, synth.tid(6, l), 1.0, "cuda") for l in range(L)]
+    ro, rl = decode_reference(q, kc, vc, bt, lens, donor, page)          # reads only positions < len
+    for b in range(B):
+        for i in range(max_pages):
+            first_dead = min(max(lens[b] - i * page, 0), page)
+            pg = int(bt[b, i])
+            kc[0][pg, :, first_dead:] = float("nan")
+            vc[0][pg, :, first_dead:] = float("nan")
+    for ns in (1, 3):
+        desc = kvp.DecodeDesc(L, B, Hq, Hkv, dh, page, max_pages, n_pages, ns)
+        ws = torch.empty(kvp.decode_workspace_bytes(desc, donor), dtype=torch.uint8, device="cuda")
+        o = [torch.full((B, Hq, dh), float("nan"), device="cuda", dtype=torch.bfloat16) for _ in range(L)]
+        lse = [torch.full((B, Hq), float("nan"), device="cuda") for _ in range(L)]
+        kvp.decode(desc, donor, q, kc, vc, bt, lengths, o, lse, ws)
+        for l in range(L):
+            close(f"o[{l}] splits={ns}", o[l], ro[l])
+            lse_close(f"lse[{l}] splits={ns}", lse[l], rl[l])
+    assert kvp.device_status() == kvp.OK
+
+
 def test_c0_prefill_then_16_decode_steps(kvp):
     """Prefill the tiny stack, move K/V into pages, then 16 decode steps: project the new token,
     append for owners, attend over the shared cache; compared step by step with the oracle run with
@@ -430,5 +468,5 @@ def test_output_projection(kvp):
         close("y", y[l], A.out_proj_fwd(f64(o[l]), f64(wo[l])))
         rd, rw = A.out_proj_bwd(f64(o[l]), f64(wo[l]), f64(dy[l]))
         close("d_o", d_o[l], rd)
-        close("dwo", dwo[l], rw)
+        close("dwo", dwo[l], rw, sum_over_tokens=True)
     assert kvp.device_status() == kvp.OK

@@ -227,6 +227,49 @@ def test_backward_vs_torch_autograd_and_group_sum_rule():
     assert dk[1] is None and dv[2] is None
 
 
+def test_selected_rows_backward_agrees_with_full_and_with_autograd():
+    """attn_bwd_rows (the row-sampled backward the full-size GPU tests call): the contributions of
+    all rows add up to the full backward; a subset of rows equals torch autograd of a loss that only
+    those rows enter; Q = 0 closed form."""
+    donor = [0, 0]
+    q, k, v = make(2, 1, 37, 4, 2, 8, donor, seed=11)
+    R = [rnd(q[0].shape, 90 + l) for l in range(2)]
+    dq, dk, dv = A.attn_bwd(q, k, v, R, donor)
+    all_rows = np.arange(37)
+    sk, sv = np.zeros((37, 8)), np.zeros((37, 8))
+    for l in range(2):
+        for hq in (2, 3):  # the two query heads of KV head 1
+            dq_r, dk_c, dv_c = A.attn_bwd_rows(q[l][0, :, hq], all_rows, k[0][0, :, 1], v[0][0, :, 1], R[l][0, :, hq])
+            assert np.allclose(dq_r, dq[l][0, :, hq], atol=1e-13)
+            sk += dk_c
+            sv += dv_c
+    assert np.allclose(sk, dk[0][0, :, 1], atol=1e-12)
+    assert np.allclose(sv, dv[0][0, :, 1], atol=1e-12)
+    # a subset of rows, non-causal and causal, against autograd of sum(R_rows * O_rows)
+    rows = np.array([0, 5, 17, 36])
+    for causal in (True, False):
+        tq = torch.from_numpy(q[1][0, :, 3].copy()).requires_grad_(True)
+        tk = torch.from_numpy(k[0][0, :, 1].copy()).requires_grad_(True)
+        tv = torch.from_numpy(v[0][0, :, 1].copy()).requires_grad_(True)
+        s = (tq @ tk.T) / math.sqrt(8)
+        if causal:
+            s = s.masked_fill(torch.triu(torch.ones(37, 37, dtype=torch.bool), 1), float("-inf"))
+        o = torch.softmax(s, dim=1) @ tv
+        (o[rows] * torch.from_numpy(R[1][0, rows, 3])).sum().backward()
+        dq_r, dk_c, dv_c = A.attn_bwd_rows(q[1][0, rows, 3], rows, k[0][0, :, 1], v[0][0, :, 1], R[1][0, rows, 3],
+                                           causal=causal)
+        assert np.allclose(dq_r, tq.grad.numpy()[rows], atol=1e-12)
+        assert np.allclose(dk_c, tk.grad.numpy(), atol=1e-12)
+        assert np.allclose(dv_c, tv.grad.numpy(), atol=1e-12)
+    # Q = 0: uniform rows, dK contribution vanishes, dV_j = sum_{i >= j} dO_i / (i + 1)
+    g = rnd((6, 3), 12)
+    kk, vv = rnd((6, 3), 13), rnd((6, 3), 14)
+    _, dk0, dv0 = A.attn_bwd_rows(np.zeros((6, 3)), np.arange(6), kk, vv, g)
+    assert np.allclose(dk0, 0.0, atol=1e-15)
+    for j in range(6):
+        assert np.allclose(dv0[j], sum(g[i] / (i + 1) for i in range(j, 6)), atol=1e-14)
+
+
 def test_backward_closed_form_zero_queries():
     donor = [0]
     _, k, v = make(1, 1, 7, 1, 1, 3, donor, seed=9)

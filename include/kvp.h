@@ -56,6 +56,15 @@ const char* kvp_status_string(int status);
  * gave up on a bounded wait since the last call (the word is cleared), or KVP_ERR_CUDA. */
 int kvp_device_status(void);
 
+/* Self-test of the bounded waits (the library's failure detection; the paper has no counterpart).  Enqueues one
+ * small GEMM in which the MMA-issuing warp withholds, once, the barrier arrival that frees a shared-memory ring
+ * stage, with a wait limit of 5 ms instead of two seconds: the TMA warp's wait for that stage runs out, it records
+ * the timeout, every other role sees the flag at its own next wait, and the kernel frees its TMEM and exits.  The
+ * call returns KVP_OK once the launch is enqueued; afterwards kvp_device_status() must return KVP_ERR_TIMEOUT
+ * (once: the word is cleared) and the device and the library remain usable.  Nothing faults and nothing spins
+ * without a limit.  scratch: DEVICE memory, 16-byte aligned, at least 512 KiB, contents irrelevant and clobbered. */
+int kvp_selftest_bounded_wait(void* scratch, size_t scratch_bytes, kvp_stream_t stream);
+
 /* Benchmark bookkeeping.  kvp_launch_count: kernels launched by this library since it was loaded.
  * kvp_set_timing_events: record the caller's CUDA events (HOST arrays of n cudaEvent_t, created by
  * the caller) immediately before and after each of the next n launches of one kernel

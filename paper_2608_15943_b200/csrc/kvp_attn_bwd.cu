@@ -54,7 +54,7 @@ constexpr int BWD_STAGES = 3;        // ring of (Q, dO) 64-row tiles
 constexpr int DQ_STAGE_BYTES = BQ2 * 32 * 4;  // one drain warp's share of a step: [64 queries x 32 columns] fp32
 // A CTA's window of query tiles is sized so that it runs about this many steps (window x streams): long enough
 // to amortise its prologue and its dK / dV reduction, short enough that a wave's footprint stays in L2.
-constexpr int kStepsPerCta = 512;
+constexpr int kStepsPerCta = 256;
 constexpr int kMinWindow = 16;
 
 template <int DH>

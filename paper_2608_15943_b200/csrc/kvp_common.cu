@@ -144,3 +144,15 @@ extern "C" int kvp_gemm(int M, int N, int K, const void* a, int64_t lda, int a_m
   return kvp::gemm_bf16(M, N, &seg, 1, a_mn ? 1 : 0, b_mn ? 1 : 0, c, ldc, out_f32 ? 1 : 0,
                         reinterpret_cast<cudaStream_t>(stream));
 }
+
+extern "C" int kvp_selftest_bounded_wait(void* scratch, size_t scratch_bytes, kvp_stream_t stream) {
+  // A [128, 512] and B [256, 512] bf16, C [128, 256] fp32; the values do not matter
+  const size_t a_bytes = 128 * 512 * 2, b_bytes = 256 * 512 * 2, c_bytes = 128 * 256 * 4;
+  if (scratch == nullptr || scratch_bytes < a_bytes + b_bytes + c_bytes || !kvp::aligned16(scratch)) return KVP_ERR_WORKSPACE;
+  uint8_t* base = reinterpret_cast<uint8_t*>(scratch);
+  kvp::GemmSeg seg{base, base + a_bytes, 512, 512, 512};
+  // eight k-blocks through a four-stage ring: the arrival that frees the first stage is withheld, so the
+  // producer's wait for that stage runs out after 5 ms
+  return kvp::gemm_bf16(128, 256, &seg, 1, 0, 0, base + a_bytes + b_bytes, 256, 1, reinterpret_cast<cudaStream_t>(stream), 1,
+                        5000000ull);
+}

@@ -36,6 +36,10 @@ struct GemmParams {
   long long ldc;
   void* c;
   uint32_t idesc;
+  // Self-test of the bounded waits (0 in every ordinary launch): the k-block count, plus one, at which the MMA
+  // warp of CTA 0 withholds the arrival that frees a ring stage, and the wait limit that launch runs with.
+  int withhold_at;
+  unsigned long long wait_limit_ns;
 };
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
@@ -107,7 +111,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           for (int kb = 0; kb < p.kblocks[seg]; ++kb, ++it) {
             const int s = it % STAGES;
             const uint32_t ph = (it / STAGES) & 1;
-            if (!mbar_wait(&empty[s], ph ^ 1, err)) { ok = false; break; }
+            if (!mbar_wait(&empty[s], ph ^ 1, err, p.wait_limit_ns)) { ok = false; break; }
             uint8_t* sa = smem + size_t(s) * STAGE_BYTES;
             uint8_t* sb = sa + A_BYTES;
             mbar_expect_tx_e(&full[s], STAGE_BYTES, leader);
@@ -142,13 +146,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
         const int acc = tile_i & 1;
         const uint32_t acc_ph = (tile_i >> 1) & 1;
-        if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1, err)) { ok = false; break; }
+        if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1, err, p.wait_limit_ns)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < total_kb; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
-          if (!mbar_wait(&full[s], ph, err)) { ok = false; break; }
+          if (!mbar_wait(&full[s], ph, err, p.wait_limit_ns)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t sa = smem_u32(smem + size_t(s) * STAGE_BYTES);
           const uint32_t sb = sa + A_BYTES;
@@ -158,7 +162,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
             const uint64_t db = smem_desc_sw128(sb + k * b_step, b_lbo, 1024);
             umma_ss(d_tmem, da, db, p.idesc, (kb | k) != 0, leader);
           }
-          umma_commit(&empty[s], leader);  // frees the smem stage once these MMAs have read it
+          // frees the smem stage once these MMAs have read it
+          if (!(p.withhold_at != 0 && blockIdx.x == 0 && it + 1 == uint32_t(p.withhold_at))) umma_commit(&empty[s], leader);
         }
         if (ok) umma_commit(&acc_full[acc], leader);
       }
@@ -172,7 +177,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       tile_coords(t, tm, tn);
       const int acc = tile_i & 1;
       const uint32_t acc_ph = (tile_i >> 1) & 1;
-      bool ok = mbar_wait(&acc_full[acc], acc_ph, err);
+      bool ok = mbar_wait(&acc_full[acc], acc_ph, err, p.wait_limit_ns);
       if (!__all_sync(0xffffffffu, ok)) break;
       tc_fence_after_sync();
       const int row = tm * BM + quarter * 32 + lane;
@@ -238,7 +243,7 @@ int gemm_read_status() {
 }
 
 int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32,
-              cudaStream_t stream) {
+              cudaStream_t stream, int withhold_at, unsigned long long wait_limit_ns) {
   if (M <= 0 || N <= 0 || nseg < 1 || nseg > MAX_SEG || c == nullptr) return KVP_ERR_INVALID_ARG;
   if ((N % 8) != 0 || (ldc % 8) != 0 || !aligned16(c)) return KVP_ERR_UNSUPPORTED;
   GemmParams p;
@@ -251,6 +256,8 @@ int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, v
   p.ldc = ldc;
   p.c = c;
   p.idesc = umma_idesc_bf16(BM, BN, a_mn, b_mn);
+  p.withhold_at = withhold_at;
+  p.wait_limit_ns = wait_limit_ns != 0 ? wait_limit_ns : kWaitLimitNs;
   for (int s = 0; s < nseg; ++s) {
     const GemmSeg& g = segs[s];
     if (g.a == nullptr || g.b == nullptr || g.K <= 0) return KVP_ERR_INVALID_ARG;
@@ -288,8 +295,9 @@ int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, v
     p.map_a[s] = p.map_a[0];
     p.map_b[s] = p.map_b[0];
   }
-  if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GEMM_SMEM)) != cudaSuccess)
-    return KVP_ERR_CUDA;
+  static const cudaError_t attr =
+      cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GEMM_SMEM));
+  if (attr != cudaSuccess) return KVP_ERR_CUDA;
   const int m_tiles = (M + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
   const int grid = min(m_tiles * n_tiles, sm_count());
   timing_before(KVP_KERNEL_GEMM, stream);

@@ -31,8 +31,9 @@ struct GemmSeg {
 //   a_mn == 0: A_s stored [M, K] row-major (K-major);  a_mn == 1: stored [K, M] row-major.
 //   b_mn == 0: B_s stored [N, K] row-major (K-major);  b_mn == 1: stored [K, N] row-major.
 //   out_f32: C is fp32 (else bf16); ldc in elements.
+// withhold_at / wait_limit_ns serve the self-test of the bounded waits (kvp_selftest_bounded_wait) only.
 int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32,
-              cudaStream_t stream);
+              cudaStream_t stream, int withhold_at = 0, unsigned long long wait_limit_ns = 0);
 
 int gemm_read_status();
 int attn_fwd_read_status();

@@ -28,7 +28,7 @@ EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_se
            "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_sim_1f1b", "kvp_workspace_bytes",
            "kvp_proj_fwd", "kvp_proj_bwd", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
            "kvp_gemm", "kvp_rmsnorm", "kvp_rope", "kvp_swiglu", "kvp_add", "kvp_decode_workspace_bytes", "kvp_cache_append",
-           "kvp_decode", "kvp_decode_static"]
+           "kvp_decode", "kvp_decode_static", "kvp_selftest_bounded_wait"]
 
 
 class KvpError(RuntimeError):
@@ -371,6 +371,17 @@ class KernelTimer:
     def durations_ms(self):
         torch.cuda.synchronize()
         return [self.starts[i].elapsed_time(self.stops[i]) for i in range(self.used)]
+
+
+lib.kvp_selftest_bounded_wait.restype = C.c_int
+lib.kvp_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+def selftest_bounded_wait(scratch: torch.Tensor):
+    """kvp_selftest_bounded_wait: enqueue the GEMM whose ring-stage arrival is withheld once; afterwards
+    device_status() returns ERR_TIMEOUT once and the library stays usable."""
+    _check(lib.kvp_selftest_bounded_wait(scratch.data_ptr(), scratch.numel() * scratch.element_size(), _stream()),
+           "kvp_selftest_bounded_wait")
 
 
 # ------------------------------------------------------------------------------------------

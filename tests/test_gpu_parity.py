@@ -12,6 +12,7 @@ import pytest
 import torch
 
 from oracle import attention as A
+from guard import Guarded
 from paper_2608_15943_b200 import synth
 from paper_2608_15943_b200 import workloads as W
 
@@ -87,12 +88,35 @@ def test_gemm_all_layouts(kvp, M, N, K, a_mn, b_mn):
         with pytest.raises(kvp.KvpError):
             kvp.gemm(sa, sb, torch.empty(M, N, device="cuda"), a_mn, b_mn)
         return
-    c32 = torch.full((M, N), float("nan"), device="cuda")
+    gd = Guarded()
+    c32 = gd.empty((M, N), torch.float32, float("nan"))
     kvp.gemm(sa, sb, c32, a_mn, b_mn)
     close("gemm f32", c32, ref, rel=1e-5, abs_=1e-4, sum_over_tokens=True)     # tight bounds, relative to |C|_inf
-    c16 = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    c16 = gd.empty((M, N), torch.bfloat16, float("nan"))
     kvp.gemm(sa, sb, c16, a_mn, b_mn)
+    gd.check()
     close("gemm bf16", c16, A.round_bf16(ref), rel=1e-3, abs_=1e-2, sum_over_tokens=True)
+    assert kvp.device_status() == kvp.OK
+
+
+def test_bounded_wait_runs_out_cleanly_and_the_library_stays_usable(kvp):
+    """Failure detection on the device: a wait that nothing satisfies gives up after its limit, the kernel
+    records the timeout, frees its TMEM and exits; the host reads the status and carries on.  The library's
+    self-test withholds one barrier arrival in a small GEMM that runs with a 5 ms limit."""
+    assert kvp.device_status() == kvp.OK
+    scratch = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    kvp.selftest_bounded_wait(scratch)
+    assert kvp.device_status() == kvp.ERR_TIMEOUT       # reported once ...
+    assert kvp.device_status() == kvp.OK                # ... and cleared
+    with pytest.raises(kvp.KvpError) as e:              # too small a scratch buffer is refused before any launch
+        kvp.selftest_bounded_wait(scratch[:1024])
+    assert e.value.status == kvp.ERR_WORKSPACE
+    # tensor memory was released and the barriers of the next launch work: an ordinary GEMM is correct
+    a = synth.normal((256, 512), 9, 1, 1.0, "cuda")
+    b = synth.normal((384, 512), 9, 2, 1.0, "cuda")
+    c = torch.full((256, 384), float("nan"), device="cuda")
+    kvp.gemm(a, b, c, 0, 0)
+    close("gemm after a timed-out launch", c, f64(a) @ f64(b).T, rel=1e-5, abs_=1e-4, sum_over_tokens=True)
     assert kvp.device_status() == kvp.OK
 
 
@@ -194,9 +218,13 @@ def test_attention_forward_and_backward_shapes(kvp, B, S, Hq, Hkv, dh, donor, ca
     L = len(donor)
     q, k, v, d_o = attn_inputs(B, S, Hq, Hkv, dh, donor)
     sh = kvp.Shape(L, B, S, 64, Hq, Hkv, dh)
-    o = [torch.full_like(x, float("nan")) for x in q]
-    lse = [torch.full((B, Hq, S), float("nan"), device="cuda") for _ in range(L)]
+    # outputs and the workspace sit between guard bands: nothing outside them may be written
+    gd = Guarded()
+    nan = float("nan")
+    o = [gd.empty(x.shape, x.dtype, nan) for x in q]
+    lse = [gd.empty((B, Hq, S), torch.float32, nan) for _ in range(L)]
     kvp.attn_fwd(sh, donor, q, k, v, o, lse, causal=causal)
+    gd.check()
     ro, rl = A.attn_fwd(f64l(q), f64l(k), f64l(v), donor, causal=causal)
     for l in range(L):
         close(f"o[{l}]", o[l], ro[l])
@@ -208,11 +236,12 @@ def test_attention_forward_and_backward_shapes(kvp, B, S, Hq, Hkv, dh, donor, ca
     for l in range(L):
         assert torch.equal(o[l], o2[l]) and torch.equal(lse[l], lse2[l])
 
-    dq = [torch.full_like(x, float("nan")) for x in q]
-    dk = [torch.full((B, S, Hkv, dh), float("nan"), device="cuda") if donor[l] == l else None for l in range(L)]
-    dv = [torch.full((B, S, Hkv, dh), float("nan"), device="cuda") if donor[l] == l else None for l in range(L)]
-    ws = torch.empty(kvp.workspace_bytes(kvp.OP_ATTN_BWD, sh, donor), dtype=torch.uint8, device="cuda")
+    dq = [gd.empty(x.shape, x.dtype, nan) for x in q]
+    dk = [gd.empty((B, S, Hkv, dh), torch.float32, nan) if donor[l] == l else None for l in range(L)]
+    dv = [gd.empty((B, S, Hkv, dh), torch.float32, nan) if donor[l] == l else None for l in range(L)]
+    ws = gd.empty((kvp.workspace_bytes(kvp.OP_ATTN_BWD, sh, donor),), torch.uint8)
     kvp.attn_bwd(sh, donor, q, k, v, o, d_o, lse, dq, dk, dv, ws, causal=causal)
+    gd.check()
     rdq, rdk, rdv = A.attn_bwd(f64l(q), f64l(k), f64l(v), f64l(d_o), donor, causal=causal)
     for l in range(L):
         close(f"dq[{l}]", dq[l], rdq[l])
@@ -297,10 +326,12 @@ def test_decode_against_oracle(kvp, L, donor, B, Hq, Hkv, dh, page, lens, ns):
     ws = torch.empty(kvp.decode_workspace_bytes(desc, donor), dtype=torch.uint8, device="cuda")
 
     def run(desc_, bt_, kc_, vc_):
-        o = [torch.full((B, Hq, dh), float("nan"), device="cuda", dtype=torch.bfloat16) for _ in range(L)]
-        lse = [torch.full((B, Hq), float("nan"), device="cuda") for _ in range(L)]
-        w = torch.empty(kvp.decode_workspace_bytes(desc_, donor), dtype=torch.uint8, device="cuda")
+        gd = Guarded()
+        o = [gd.empty((B, Hq, dh), torch.bfloat16, float("nan")) for _ in range(L)]
+        lse = [gd.empty((B, Hq), torch.float32, float("nan")) for _ in range(L)]
+        w = gd.empty((kvp.decode_workspace_bytes(desc_, donor),), torch.uint8)
         kvp.decode(desc_, donor, q, kc_, vc_, bt_, lengths, o, lse, w)
+        gd.check()
         return o, lse
 
     o, lse = run(desc, bt, kc, vc)

@@ -9,17 +9,20 @@ It restates, in Python integers (arbitrary precision, so no rounding anywhere):
            the stage totals, the LM head counted on the last stage.  Kept as the
            exact rational (max_i F_i * P) / (sum_i F_i).
 * Eq. 6-7  stage totals under a conversion mask z and the budget sum z <= m.
-* Algorithm 1 (Architecture-Balanced KV-Pipe), step by step in the paper's
-  order: start at the tail stage; once the tail is within (1+eps) of the
-  average retarget to the arg-max stage; convert the deepest unconverted layer
-  of the chosen stage; stop on FIR <= 1+eps, on the budget, or when the chosen
-  stage has no convertible layer.
+* Algorithm 1 (Architecture-Balanced KV-Pipe): start at the tail stage; once
+  the tail is within (1+eps) of the average retarget to the arg-max stage;
+  convert the deepest unconverted layer of the chosen stage; stop on
+  FIR <= 1+eps, on the budget, or when the chosen stage has no convertible
+  layer.  The state is the set of converted layers and every quantity is
+  recomputed from Eq. 4-7 each round.
 * Appendix "Optional Safe-Layer Guardrail": only layers with (1-indexed)
   l >= ceil(alpha L) are admissible.
 * Appendix "Attention FLOPs under MHA and GQA": per-token forward FLOPs and the
   saving 4 h^2 / r of a converted layer.
 * The Uniform and Symmetric-Bipolar placements of the stage tables in the
-  appendix "Stage-level splits".
+  appendix "Stage-level splits".  The paper gives each a sentence and one
+  stage table (m = 4, P = 8); how they continue beyond that instance (more
+  conversions than stages, a full stage) is this build's definition.
 
 Readings where the paper is silent (each is also a documented reading of the
 library): tau(l) is the nearest preceding unconverted layer; global layer 0 is
@@ -103,49 +106,63 @@ def _admissible(l, stage_begin, i, L, alpha, stage_local_donor):
 
 def kvp_plan(stage_begin, f_full, f_share, stage_extra, eps=(0, 1), max_conv=0,
              stop_on_no_improve=False, stage_local_donor=False, alpha=None):
-    """Algorithm 1.  eps = (num, den) rational; max_conv 0 means L.
+    """Algorithm 1 (Architecture-Balanced KV-Pipe).  eps = (num, den) rational; max_conv 0 means L.
+
+    Stated through the paper's definitions rather than through incremental bookkeeping: the state is the SET of
+    converted layers; every round recomputes the stage totals of that set from Eq. 6 and the imbalance from
+    Eq. 4-5, then
+      * stops if FIR <= 1 + eps, or if the budget sum z = m of Eq. 7 is spent;
+      * targets the tail stage while the tail is still heavier than (1 + eps) times the average stage, and
+        otherwise the heaviest stage (the deepest one among equals);
+      * converts the deepest layer of the target stage that is still unconverted and admissible, or stops if
+        there is none;
+      * under the optional no-improve rule, keeps the conversion only if the FIR of the enlarged set is strictly
+        smaller.
+    All comparisons are between exact integer cross-products.
 
     Returns dict(z, donor, stage, fir_num, fir_den, n_conv, stop_reason)."""
     P = len(stage_begin) - 1
     L = stage_begin[P]
-    m = max_conv if max_conv else L
+    budget = max_conv if max_conv else L
     en, ed = eps
-    z = [0] * L
-    stage = stage_totals(stage_begin, f_full, f_share, stage_extra, z)   # line 2
-    t = 0
-    reason = STOP_TOLERANCE
+
+    def totals(converted):
+        return stage_totals(stage_begin, f_full, f_share, stage_extra, [int(l in converted) for l in range(L)])
+
+    def above_tolerance(value_times_p, total):        # value / (total / P) > 1 + eps
+        return value_times_p * ed > (ed + en) * total
+
+    converted = set()
     while True:
-        num, den = fir_rational(stage)                                   # line 3 / 15
-        if not (num * ed > (ed + en) * den):      # FIR > 1 + eps ?
+        stage = totals(converted)
+        num, den = fir_rational(stage)
+        if not above_tolerance(num, den):
             reason = STOP_TOLERANCE
             break
-        if not (t < m):
+        if len(converted) >= budget:
             reason = STOP_BUDGET
             break
-        i_star = P - 1                                                    # line 7
-        if stage[i_star] * P * ed <= (ed + en) * den:                     # line 8
-            mx = max(stage)
-            i_star = max(j for j in range(P) if stage[j] == mx)           # line 9
-        cand = [l for l in range(stage_begin[i_star], stage_begin[i_star + 1])
-                if not z[l] and _admissible(l, stage_begin, i_star, L, alpha, stage_local_donor)]
-        if not cand:                                                      # line 12
+        if above_tolerance(stage[P - 1] * P, den):
+            target = P - 1
+        else:
+            target = max(range(P), key=lambda j: (stage[j], j))
+        pool = {l for l in range(stage_begin[target], stage_begin[target + 1])
+                if l not in converted and _admissible(l, stage_begin, target, L, alpha, stage_local_donor)}
+        if not pool:
             reason = STOP_EXHAUSTED
             break
-        l_star = max(cand)                                                # line 11
-        delta = f_full[l_star] - f_share[l_star]                          # line 16
+        pick = max(pool)
         if stop_on_no_improve:
-            trial = list(stage)
-            trial[i_star] -= delta
-            n2, d2 = fir_rational(trial)
-            if not (n2 * den < num * d2):        # FIR(after) < FIR(before) ?
+            num_after, den_after = fir_rational(totals(converted | {pick}))
+            if not (num_after * den < num * den_after):
                 reason = STOP_NO_IMPROVE
                 break
-        z[l_star] = 1                                                     # line 15
-        stage[i_star] -= delta                                            # line 17
-        t += 1                                                            # line 18
+        converted.add(pick)
+    z = [int(l in converted) for l in range(L)]
+    stage = totals(converted)
     num, den = fir_rational(stage)
     return dict(z=z, donor=donor_from_z(z), stage=stage, fir_num=num, fir_den=den,
-                n_conv=t, stop_reason=reason)
+                n_conv=len(converted), stop_reason=reason)
 
 
 def exhaustive_min_fir(stage_begin, f_full, f_share, stage_extra, max_conv=0):

@@ -11,92 +11,91 @@ namespace {
 
 typedef unsigned __int128 u128;
 
-struct Fir {
-  uint64_t num;  // max_i F_i * P
-  uint64_t den;  // sum_i F_i
+// The planner's working state: per-stage totals (Eq. 6) kept incrementally with their sum, and for every stage
+// the index below which its layers are still unconverted (conversions inside a stage always go deepest-first,
+// so the converted layers of a stage form a suffix of it).
+struct PlanState {
+  const kvp_plan_in* in;
+  int L, P;
+  std::vector<uint64_t> total;   // F_stage_i(z)
+  u128 sum;                      // sum_i F_stage_i(z)
+  std::vector<int> frontier;     // stage i: layers [frontier[i], stage_begin[i+1]) are converted
+  int lowest_admissible;         // smallest layer index the guardrail and "never layer 0" admit
+
+  uint64_t saving(int l) const { return in->f_full[l] - in->f_share[l]; }
+  uint64_t heaviest() const { return *std::max_element(total.begin(), total.end()); }
+
+  // deepest layer of stage i that Algorithm 1 may still convert, or -1
+  int candidate(int i) const {
+    const int l = frontier[i] - 1;
+    int floor_l = std::max(in->stage_begin[i], lowest_admissible);
+    if ((in->flags & KVP_PLAN_STAGE_LOCAL_DONOR) && floor_l == in->stage_begin[i]) ++floor_l;
+    return l >= floor_l ? l : -1;
+  }
+  void convert(int i, uint8_t* z) {
+    const int l = --frontier[i];
+    z[l] = 1;
+    total[i] -= saving(l);
+    sum -= saving(l);
+  }
 };
 
-bool stage_sums_fit(const std::vector<uint64_t>& stage) {
-  u128 sum = 0, mx = 0;
-  for (uint64_t f : stage) {
-    sum += f;
-    if (f > mx) mx = f;
+// value / (sum / P) > 1 + en/ed, in integers
+bool above_tolerance(u128 value, int P, u128 sum, u128 en, u128 ed) { return value * u128(P) * ed > (ed + en) * sum; }
+
+// Uniform placement: rounds over the stages from the last one leftwards, one conversion per stage and round,
+// until m are placed.  In closed form: stage i, which can give up cap_i layers, takes min(cap_i, R) in the R
+// complete rounds that fit and one more if it is among the first stages (from the right) of the partial round.
+void place_uniform(PlanState& st, uint8_t* z, int m) {
+  const int P = st.P;
+  std::vector<int> cap(P), take(P, 0);
+  int64_t all = 0;
+  for (int i = 0; i < P; ++i) {
+    cap[i] = st.in->stage_begin[i + 1] - std::max(st.in->stage_begin[i], 1);   // layer 0 is never converted
+    all += cap[i];
   }
-  const u128 lim = ~uint64_t(0);
-  return sum <= lim && mx * stage.size() <= lim;
-}
-
-Fir fir_of(const std::vector<uint64_t>& stage) {
-  uint64_t mx = 0, sum = 0;
-  for (uint64_t f : stage) {
-    sum += f;
-    if (f > mx) mx = f;
+  const int64_t want = std::min<int64_t>(m, all);
+  const int deepest_stage = *std::max_element(cap.begin(), cap.end());
+  int rounds = 0;
+  while (rounds < deepest_stage) {   // the largest R whose complete rounds place no more than `want`
+    int64_t placed = 0;
+    for (int i = 0; i < P; ++i) placed += std::min(cap[i], rounds + 1);
+    if (placed > want) break;
+    ++rounds;
   }
-  return Fir{mx * uint64_t(stage.size()), sum};
-}
-
-// a/b > c/d for positive denominators
-bool frac_gt(u128 a, u128 b, u128 c, u128 d) { return a * d > c * b; }
-
-bool admissible(int l, int stage_first, const kvp_plan_in* in) {
-  if (l == 0) return false;
-  if ((in->flags & KVP_PLAN_STAGE_LOCAL_DONOR) && l == stage_first) return false;
-  if (in->alpha_num != 0) {
-    // 1-indexed layer l+1 must satisfy l+1 >= ceil(alpha * L)
-    const uint64_t need = (uint64_t(in->alpha_num) * uint64_t(in->L) + in->alpha_den - 1) / in->alpha_den;
-    if (uint64_t(l) + 1 < need) return false;
+  int64_t left = want;
+  for (int i = 0; i < P; ++i) {
+    take[i] = std::min(cap[i], rounds);
+    left -= take[i];
   }
-  return true;
-}
-
-int deepest_convertible(const kvp_plan_in* in, const uint8_t* z, int stage) {
-  const int first = in->stage_begin[stage], last = in->stage_begin[stage + 1];
-  for (int l = last - 1; l >= first; --l)
-    if (!z[l] && admissible(l, first, in)) return l;
-  return -1;
-}
-
-// deepest unconverted layer of a stage for the comparison placements (only layer 0 is excluded)
-int deepest_plain(const kvp_plan_in* in, const uint8_t* z, int stage) {
-  for (int l = in->stage_begin[stage + 1] - 1; l >= in->stage_begin[stage]; --l)
-    if (!z[l] && l > 0) return l;
-  return -1;
-}
-
-void place_uniform(const kvp_plan_in* in, uint8_t* z, int m) {
-  const int P = in->P;
-  int i = P - 1, t = 0, idle = 0;
-  while (t < m && idle < P) {
-    const int l = deepest_plain(in, z, i);
-    if (l >= 0) {
-      z[l] = 1;
-      ++t;
-      idle = 0;
-    } else {
-      ++idle;
+  for (int i = P - 1; i >= 0 && left > 0; --i)
+    if (cap[i] > rounds) {
+      ++take[i];
+      --left;
     }
-    i = i > 0 ? i - 1 : P - 1;
-  }
+  for (int i = 0; i < P; ++i)
+    for (int k = 0; k < take[i]; ++k) st.convert(i, z);
 }
 
-void place_bipolar(const kvp_plan_in* in, uint8_t* z, int m) {
-  const int P = in->P;
-  int anchors[2] = {P - 1, P / 2 - 1 > 0 ? P / 2 - 1 : 0};
-  int t = 0, turn = 0, idle = 0;
-  while (t < m && idle < 2 * P) {
-    const int a = turn % 2;
-    const int i = anchors[a];
-    const int l = i >= 0 ? deepest_plain(in, z, i) : -1;
-    if (l >= 0) {
-      z[l] = 1;
-      ++t;
-      idle = 0;
-      ++turn;
-    } else {
-      anchors[a] -= 1;
-      ++idle;
-      if (anchors[a] < 0) ++turn;
-    }
+// Symmetric-Bipolar placement: two cursors, one starting at the deepest layer of the last stage and one at the
+// deepest layer of the middle stage (index P/2 - 1), take turns; a cursor converts the deepest unconverted
+// layer at or below its position and, stages being contiguous, simply walks down the layer indices; a cursor
+// that has run past layer 1 loses its turns.
+void place_bipolar(PlanState& st, uint8_t* z, int m) {
+  const int P = st.P;
+  const int mid = std::max(P / 2 - 1, 0);
+  int cursor[2] = {st.L - 1, st.in->stage_begin[mid + 1] - 1};
+  std::vector<int> stage_of(st.L);
+  for (int i = 0; i < P; ++i)
+    for (int l = st.in->stage_begin[i]; l < st.in->stage_begin[i + 1]; ++l) stage_of[l] = i;
+  int placed = 0;
+  for (int turn = 0; placed < m && (cursor[0] >= 1 || cursor[1] >= 1); ++turn) {
+    int& c = cursor[turn & 1];
+    while (c >= 1 && z[c]) --c;
+    if (c < 1) continue;
+    // within a stage conversions are deepest-first for both cursors, so c is that stage's frontier layer
+    st.convert(stage_of[c], z);
+    ++placed;
   }
 }
 
@@ -130,89 +129,94 @@ extern "C" int kvp_plan(const kvp_plan_in* in, kvp_plan_out* out) {
 
   uint8_t* z = out->z;
   for (int l = 0; l < L; ++l) z[l] = 0;
-  std::vector<uint64_t> stage(P);
-  {
-    std::vector<u128> wide(P);
-    for (int i = 0; i < P; ++i) {
-      wide[i] = in->stage_extra[i];
-      for (int l = in->stage_begin[i]; l < in->stage_begin[i + 1]; ++l) wide[i] += in->f_full[l];
-      if (wide[i] > u128(~uint64_t(0))) return KVP_ERR_UNSUPPORTED;
-      stage[i] = uint64_t(wide[i]);
-    }
+  PlanState st;
+  st.in = in;
+  st.L = L;
+  st.P = P;
+  st.total.resize(P);
+  st.frontier.resize(P);
+  st.sum = 0;
+  for (int i = 0; i < P; ++i) {
+    u128 wide = in->stage_extra[i];
+    for (int l = in->stage_begin[i]; l < in->stage_begin[i + 1]; ++l) wide += in->f_full[l];
+    if (wide > u128(~uint64_t(0))) return KVP_ERR_UNSUPPORTED;
+    st.total[i] = uint64_t(wide);
+    st.sum += wide;
+    st.frontier[i] = in->stage_begin[i + 1];
   }
-  if (!stage_sums_fit(stage)) return KVP_ERR_UNSUPPORTED;
+  // the exact fraction max * P / sum is returned in 64-bit words
+  if (st.sum > u128(~uint64_t(0)) || u128(st.heaviest()) * u128(P) > u128(~uint64_t(0))) return KVP_ERR_UNSUPPORTED;
+  st.lowest_admissible = 1;
+  if (in->alpha_num != 0) {
+    // 1-indexed layer l+1 >= ceil(alpha L)  <=>  l >= ceil(alpha L) - 1
+    const uint64_t need = (uint64_t(in->alpha_num) * uint64_t(L) + in->alpha_den - 1) / in->alpha_den;
+    st.lowest_admissible = std::max<int>(1, int(need) - 1);
+  }
 
-  const int m = in->max_conv ? in->max_conv : L;
+  const int budget = in->max_conv ? in->max_conv : L;
   const u128 en = in->eps_num, ed = in->eps_den;
-  int t = 0;
-  int reason = KVP_STOP_TOLERANCE;
+  int reason = KVP_STOP_BUDGET;
+  int n_conv = 0;
 
-  if (in->placement == KVP_PLACE_UNIFORM || in->placement == KVP_PLACE_BIPOLAR) {
-    if (in->placement == KVP_PLACE_UNIFORM) place_uniform(in, z, m); else place_bipolar(in, z, m);
-    for (int i = 0; i < P; ++i)
-      for (int l = in->stage_begin[i]; l < in->stage_begin[i + 1]; ++l)
-        if (z[l]) {
-          stage[i] -= in->f_full[l] - in->f_share[l];
-          ++t;
-        }
-    reason = KVP_STOP_BUDGET;
+  if (in->placement == KVP_PLACE_UNIFORM) {
+    place_uniform(st, z, budget);
+  } else if (in->placement == KVP_PLACE_BIPOLAR) {
+    place_bipolar(st, z, budget);
   } else if (in->placement == KVP_PLACE_ARCH_BALANCED) {
     for (;;) {
-      const Fir f = fir_of(stage);
-      if (!(u128(f.num) * ed > (ed + en) * u128(f.den))) {  // FIR <= 1 + eps
+      const uint64_t top = st.heaviest();
+      if (!above_tolerance(top, P, st.sum, en, ed)) {
         reason = KVP_STOP_TOLERANCE;
         break;
       }
-      if (!(t < m)) {
+      if (n_conv >= budget) {
         reason = KVP_STOP_BUDGET;
         break;
       }
-      int i_star = P - 1;  // the tail stage
-      if (u128(stage[i_star]) * uint64_t(P) * ed <= (ed + en) * u128(f.den)) {
-        uint64_t mx = 0;
-        for (int j = 0; j < P; ++j)
-          if (stage[j] >= mx) {  // ties -> highest stage index
-            mx = stage[j];
-            i_star = j;
-          }
-      }
-      const int l_star = deepest_convertible(in, z, i_star);
-      if (l_star < 0) {
+      // the tail stage while it is still too heavy, otherwise the heaviest stage, the deepest among equals
+      int target = P - 1;
+      if (!above_tolerance(st.total[target], P, st.sum, en, ed))
+        for (int j = P - 1; j >= 0; --j)
+          if (st.total[j] > st.total[target]) target = j;
+      const int l = st.candidate(target);
+      if (l < 0) {
         reason = KVP_STOP_EXHAUSTED;
         break;
       }
-      const uint64_t delta = in->f_full[l_star] - in->f_share[l_star];
       if (in->flags & KVP_PLAN_STOP_ON_NO_IMPROVE) {
-        std::vector<uint64_t> trial(stage);
-        trial[i_star] -= delta;
-        const Fir g = fir_of(trial);
-        if (!frac_gt(f.num, f.den, g.num, g.den)) {  // FIR would not strictly drop
+        // FIR after the conversion: the new maximum is the lighter target or the heaviest of the others
+        uint64_t top_after = st.total[target] - st.saving(l);
+        for (int j = 0; j < P; ++j)
+          if (j != target && st.total[j] > top_after) top_after = st.total[j];
+        const u128 sum_after = st.sum - st.saving(l);
+        if (!(u128(top_after) * st.sum < u128(top) * sum_after)) {   // top_after/sum_after < top/sum ?
           reason = KVP_STOP_NO_IMPROVE;
           break;
         }
       }
-      z[l_star] = 1;
-      stage[i_star] -= delta;
-      ++t;
+      st.convert(target, z);
+      ++n_conv;
     }
   } else {
     return KVP_ERR_INVALID_ARG;
   }
+  if (in->placement != KVP_PLACE_ARCH_BALANCED)
+    for (int l = 0; l < L; ++l) n_conv += z[l];
 
   int last_owner = -1;
   for (int l = 0; l < L; ++l) {
     if (!z[l]) last_owner = l;
     out->donor[l] = last_owner;
   }
-  const Fir f = fir_of(stage);
+  const uint64_t top = st.heaviest();
   for (int i = 0; i < P; ++i) {
-    out->stage_flops[i] = stage[i];
-    out->stage_ratio[i] = double(stage[i]) * double(P) / double(f.den);
+    out->stage_flops[i] = st.total[i];
+    out->stage_ratio[i] = double(st.total[i]) * double(P) / double(uint64_t(st.sum));
   }
-  out->fir_num = f.num;
-  out->fir_den = f.den;
-  out->fir = double(f.num) / double(f.den);
-  out->n_conv = t;
+  out->fir_num = top * uint64_t(P);
+  out->fir_den = uint64_t(st.sum);
+  out->fir = double(out->fir_num) / double(out->fir_den);
+  out->n_conv = n_conv;
   out->stop_reason = reason;
   return KVP_OK;
 }

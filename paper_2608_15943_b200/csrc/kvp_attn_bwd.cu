@@ -27,6 +27,7 @@
 #include <math.h>
 
 #include <algorithm>
+#include <vector>
 
 #include "kvp_host.h"
 #include "kvp_sm100.cuh"
@@ -75,20 +76,25 @@ struct BwdSmem {
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
 
+// One launch serves several donor groups (up to MAX_GROUP member layers in all): slot i of the per-layer arrays is
+// the i-th member layer, group g owns slots [first_slot[g], first_slot[g + 1]) and blocks [cta_begin[g],
+// cta_begin[g + 1]).  Groups are sorted by size, largest first, so that only the last, shortest CTAs of the whole
+// backward pass run on a partly idle device.
 struct BwdParams {
-  CUtensorMap map_k, map_v;       // donor K, V: [B,S,Hkv,dh], box rows 128
-  CUtensorMap map_q[MAX_GROUP];   // per layer of the group, box rows 64
-  CUtensorMap map_do[MAX_GROUP];
+  CUtensorMap map_k[MAX_GROUP], map_v[MAX_GROUP];   // per group: donor K, V [B,S,Hkv,dh], box rows 128
+  CUtensorMap map_q[MAX_GROUP], map_do[MAX_GROUP];  // per member layer, box rows 64
   const float* lse[MAX_GROUP];    // [B,Hq,S]
   const float* delta[MAX_GROUP];  // [B,Hq,S]
   float* dq_acc[MAX_GROUP];       // blocked fp32 accumulators, see dq_acc_floats()
-  float* dk_sum;                  // fp32 [B,S,Hkv,dh]
-  float* dv_sum;
-  int n_layers;
+  float* dk_sum[MAX_GROUP];       // per group: fp32 [B,S,Hkv,dh]
+  float* dv_sum[MAX_GROUP];
+  int first_slot[MAX_GROUP + 1];
+  int cta_begin[MAX_GROUP + 1];
+  int window[MAX_GROUP];          // query tiles per CTA
+  int ctas_per_pair[MAX_GROUP];   // CTAs of one (batch, KV head): sum over windows of the key tiles that see the window
+  int n_groups;
   int B, S, Hq, Hkv;
   int causal;
-  int window;                     // query tiles per CTA
-  int ctas_per_pair;              // CTAs of one (batch, KV head): sum over windows of the key tiles that see the window
   float scale;
   float scale_log2;
 };
@@ -152,7 +158,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
   const int lane = threadIdx.x & 31;
   int* err = &g_bwd_status;
 
-  // Work decomposition.  A CTA is one (batch, KV head), one 128-row key tile and one WINDOW of p.window
+  // Work decomposition.  A CTA is one donor group, one (batch, KV head), one 128-row key tile and one WINDOW of
   // consecutive 64-row query tiles, for every query stream of the donor group.  All CTAs therefore take
   // (nearly) the same number of steps per stream and walk the streams at the same pace, so the CTAs that
   // run at the same time read the same few Q / dO tiles and add to the same few dQ accumulator tiles:
@@ -161,11 +167,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
   // dK / dV partials to the (cleared) output with reductions.
   const int n_jt = (p.S + BT - 1) / BT;
   const int n_qt = (p.S + BQ2 - 1) / BQ2;
-  const int pair = blockIdx.x / p.ctas_per_pair;
-  int jt = blockIdx.x - pair * p.ctas_per_pair;
+  int grp = 0;
+  while (grp + 1 < p.n_groups && int(blockIdx.x) >= p.cta_begin[grp + 1]) ++grp;
+  const int slot0 = p.first_slot[grp];
+  const int n_layers = p.first_slot[grp + 1] - slot0;
+  const int window = p.window[grp];
+  const int in_group = blockIdx.x - p.cta_begin[grp];
+  const int pair = in_group / p.ctas_per_pair[grp];
+  int jt = in_group - pair * p.ctas_per_pair[grp];
   int win = 0;
   for (;; ++win) {
-    const int vis = p.causal ? min(n_jt, ((win + 1) * p.window * BQ2 + BT - 1) / BT) : n_jt;
+    const int vis = p.causal ? min(n_jt, ((win + 1) * window * BQ2 + BT - 1) / BT) : n_jt;
     if (jt < vis) break;
     jt -= vis;
   }
@@ -173,9 +185,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
   const int b = pair / p.Hkv;
   const int G = p.Hq / p.Hkv;
   const int kv0 = jt * BT;
-  const int qt_first = max(p.causal ? (kv0 / BQ2) : 0, win * p.window);
-  const int per_stream = min(n_qt, (win + 1) * p.window) - qt_first;
-  const int n_iter = p.n_layers * G * per_stream;
+  const int qt_first = max(p.causal ? (kv0 / BQ2) : 0, win * window);
+  const int per_stream = min(n_qt, (win + 1) * window) - qt_first;
+  const int n_iter = n_layers * G * per_stream;
 
   if (threadIdx.x == 0) {
     mbar_init(kv_full, 1);
@@ -224,13 +236,13 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
     // ------------------------------ TMA producer ------------------------------
     {
       const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
-      if (leader) tma_prefetch_desc(&p.map_k);
-      if (leader) tma_prefetch_desc(&p.map_v);
+      if (leader) tma_prefetch_desc(&p.map_k[grp]);
+      if (leader) tma_prefetch_desc(&p.map_v[grp]);
       mbar_expect_tx_e(kv_full, 2 * L::KV_TILE, leader);
 #pragma unroll
       for (int h = 0; h < HALVES; ++h) {
-        tma_load_4d_e(smem + L::OFF_K + h * HALF_BYTES, &p.map_k, kv_full, h * 64, hk, kv0, b, leader);
-        tma_load_4d_e(smem + L::OFF_V + h * HALF_BYTES, &p.map_v, kv_full, h * 64, hk, kv0, b, leader);
+        tma_load_4d_e(smem + L::OFF_K + h * HALF_BYTES, &p.map_k[grp], kv_full, h * 64, hk, kv0, b, leader);
+        tma_load_4d_e(smem + L::OFF_V + h * HALF_BYTES, &p.map_v[grp], kv_full, h * 64, hk, kv0, b, leader);
       }
       for (int it = 0; it < n_iter; ++it) {
         int li, hq, q0;
@@ -242,8 +254,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
         uint8_t* dst = smem + L::OFF_RING + s * L::STAGE;
 #pragma unroll
         for (int h = 0; h < HALVES; ++h) {
-          tma_load_4d_e(dst + h * QHALF_BYTES, &p.map_q[li], &q_full[s], h * 64, hq, q0, b, leader);
-          tma_load_4d_e(dst + L::Q_TILE + h * QHALF_BYTES, &p.map_do[li], &q_full[s], h * 64, hq, q0, b, leader);
+          tma_load_4d_e(dst + h * QHALF_BYTES, &p.map_q[slot0 + li], &q_full[s], h * 64, hq, q0, b, leader);
+          tma_load_4d_e(dst + L::Q_TILE + h * QHALF_BYTES, &p.map_do[slot0 + li], &q_full[s], h * 64, hq, q0, b, leader);
         }
       }
     }
@@ -359,7 +371,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
       const float* row = nullptr;
     };
     auto row_of = [&](int li, int g) {
-      const float* src = stat_kind == 0 ? p.lse[li < p.n_layers ? li : 0] : p.delta[li < p.n_layers ? li : 0];
+      const int slot = slot0 + (li < n_layers ? li : 0);
+      const float* src = stat_kind == 0 ? p.lse[slot] : p.delta[slot];
       return src + (size_t(b) * p.Hq + hk * G + g) * p.S;
     };
     auto advance = [&](Cursor& c) {
@@ -481,7 +494,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
       // warpgroup 0 adds dK (scaled), warpgroup 1 adds dV; every lane loads, valid rows reduce
       const bool valid = kv_row < p.S;
       const size_t row_off = ((size_t(b) * p.S + (valid ? kv_row : 0)) * p.Hkv + hk) * DH;
-      float* dst = (wg == 0 ? p.dk_sum : p.dv_sum) + row_off;
+      float* dst = (wg == 0 ? p.dk_sum[grp] : p.dv_sum[grp]) + row_off;
       const uint32_t src = (wg == 0 ? tm_dk : tm_dv) + lane_sel;
       const float mul = wg == 0 ? p.scale : 1.f;
 #pragma unroll 1
@@ -523,7 +536,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
       mbar_arrive(dq_free);
       if (active) {
         const size_t tile = ((size_t(b) * p.Hq + hk * G + g) * n_qt + (qt_first + qi)) * (DH / 32) + quarter;
-        float* dst = p.dq_acc[li] + tile * (BQ2 * 32);
+        float* dst = p.dq_acc[slot0 + li] + tile * (BQ2 * 32);
         // the previous step's reduction has read the buffer
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncwarp();
@@ -654,16 +667,9 @@ int make_map_bshd(CUtensorMap* m, const void* base, int B, int S, int H, int dh,
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
-int largest_group(const kvp_shape* s, const int32_t* donor) {
-  int best = 1;
-  for (int d = 0; d < s->L; ++d) {
-    if (donor[d] != d) continue;
-    int n = 0;
-    for (int l = d; l < s->L; ++l) n += donor[l] == d;
-    best = n > best ? n : best;
-  }
-  return best;
-}
+// Member layers of the launches' accumulators that are live at once: a launch takes whole donor groups until it
+// holds MAX_GROUP member layers.
+int max_layers_per_launch(const kvp_shape* s) { return s->L < MAX_GROUP ? s->L : MAX_GROUP; }
 
 }  // namespace
 
@@ -677,12 +683,12 @@ int attn_bwd_read_status() {
   return v;
 }
 
-// Workspace: Delta [B,Hq,S] fp32 for every layer, then the fp32 dQ accumulators of the largest donor group
-// (one per member layer; groups are processed one after the other and reuse them).
+// Workspace: Delta [B,Hq,S] fp32 for every layer, then the fp32 dQ accumulators of the member layers of one launch
+// (launches run one after the other and reuse them).
 size_t attn_bwd_workspace(const kvp_shape* s, const int32_t* donor) {
-  const int n = donor != nullptr ? largest_group(s, donor) : s->L;
+  (void)donor;
   return size_t(s->L) * align256(size_t(s->B) * s->Hq * s->S * 4) +
-         size_t(n > MAX_GROUP ? MAX_GROUP : n) * align256(dq_acc_floats(s->B, s->S, s->Hq, s->dh) * 4);
+         size_t(max_layers_per_launch(s)) * align256(dq_acc_floats(s->B, s->S, s->Hq, s->dh) * 4);
 }
 
 int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
@@ -722,33 +728,82 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
   timing_after(KVP_KERNEL_ATTN_BWD_AUX, stream);
   if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
 
-  // One launch per donor group: dK / dV of the donor (written, not added to: a donor shared by more than
-  // MAX_GROUP layers is not supported) and the dQ accumulators of every member layer.
+  // Donor groups, largest first; a launch takes groups until it holds MAX_GROUP member layers.  A launch writes
+  // dK / dV of its donors through reductions into cleared buffers, so a donor shared by more than MAX_GROUP
+  // layers is not supported.
+  struct Group {
+    int owner, n;
+    int members[MAX_GROUP];
+  };
+  std::vector<Group> groups;
   for (int d = 0; d < s->L; ++d) {
     if (donor[d] != d) continue;
-    int members[MAX_GROUP];
-    int n = 0;
+    Group g;
+    g.owner = d;
+    g.n = 0;
     for (int l = d; l < s->L; ++l)
       if (donor[l] == d) {
-        if (n == MAX_GROUP) return KVP_ERR_UNSUPPORTED;
-        members[n++] = l;
+        if (g.n == MAX_GROUP) return KVP_ERR_UNSUPPORTED;
+        g.members[g.n++] = l;
       }
+    groups.push_back(g);
+  }
+  std::stable_sort(groups.begin(), groups.end(), [](const Group& a, const Group& b) { return a.n > b.n; });
+  const int n_jt = (s->S + BT - 1) / BT, n_qt = (s->S + BQ2 - 1) / BQ2, n_pairs = s->Hkv * s->B;
+  const int G = s->Hq / s->Hkv;
+  const size_t kv_bytes = size_t(s->B) * s->S * s->Hkv * dh * 4;
+  size_t gi = 0;
+  while (gi < groups.size()) {
     BwdParams p;
-    int rc = make_map_bshd(&p.map_k, k[d], s->B, s->S, s->Hkv, dh, BT);
-    if (rc == KVP_OK) rc = make_map_bshd(&p.map_v, v[d], s->B, s->S, s->Hkv, dh, BT);
-    if (rc != KVP_OK) return rc;
-    for (int i = 0; i < MAX_GROUP; ++i) {
-      const int l = members[i < n ? i : 0];
-      rc = make_map_bshd(&p.map_q[i], q[l], s->B, s->S, s->Hq, dh, BQ2);
-      if (rc == KVP_OK) rc = make_map_bshd(&p.map_do[i], d_o[l], s->B, s->S, s->Hq, dh, BQ2);
+    int slots = 0, ng = 0;
+    int slot_layer[MAX_GROUP];
+    p.cta_begin[0] = 0;
+    p.first_slot[0] = 0;
+    while (gi < groups.size() && slots + groups[gi].n <= MAX_GROUP) {
+      const Group& g = groups[gi];
+      int rc = make_map_bshd(&p.map_k[ng], k[g.owner], s->B, s->S, s->Hkv, dh, BT);
+      if (rc == KVP_OK) rc = make_map_bshd(&p.map_v[ng], v[g.owner], s->B, s->S, s->Hkv, dh, BT);
       if (rc != KVP_OK) return rc;
-      p.lse[i] = lse[l];
-      p.delta[i] = reinterpret_cast<const float*>(wsb + size_t(l) * delta_bytes);
-      p.dq_acc[i] = reinterpret_cast<float*>(acc_base + size_t(i < n ? i : 0) * acc_bytes);
+      for (int i = 0; i < g.n; ++i) {
+        const int l = g.members[i];
+        rc = make_map_bshd(&p.map_q[slots], q[l], s->B, s->S, s->Hq, dh, BQ2);
+        if (rc == KVP_OK) rc = make_map_bshd(&p.map_do[slots], d_o[l], s->B, s->S, s->Hq, dh, BQ2);
+        if (rc != KVP_OK) return rc;
+        p.lse[slots] = lse[l];
+        p.delta[slots] = reinterpret_cast<const float*>(wsb + size_t(l) * delta_bytes);
+        p.dq_acc[slots] = reinterpret_cast<float*>(acc_base + size_t(slots) * acc_bytes);
+        slot_layer[slots] = l;
+        ++slots;
+      }
+      p.dk_sum[ng] = dk_sum[g.owner];
+      p.dv_sum[ng] = dv_sum[g.owner];
+      p.window[ng] = std::min(n_qt, std::max(kMinWindow, (kStepsPerCta + g.n * G - 1) / (g.n * G)));
+      p.ctas_per_pair[ng] = 0;
+      for (int w = 0; w * p.window[ng] < n_qt; ++w)
+        p.ctas_per_pair[ng] += causal ? std::min(n_jt, ((w + 1) * p.window[ng] * BQ2 + BT - 1) / BT) : n_jt;
+      p.first_slot[ng + 1] = slots;
+      p.cta_begin[ng + 1] = p.cta_begin[ng] + n_pairs * p.ctas_per_pair[ng];
+      ++ng;
+      ++gi;
     }
-    p.dk_sum = dk_sum[d];
-    p.dv_sum = dv_sum[d];
-    p.n_layers = n;
+    for (int i = slots; i < MAX_GROUP; ++i) {   // unused entries repeat slot 0, so that no descriptor is left unset
+      p.map_q[i] = p.map_q[0];
+      p.map_do[i] = p.map_do[0];
+      p.lse[i] = p.lse[0];
+      p.delta[i] = p.delta[0];
+      p.dq_acc[i] = p.dq_acc[0];
+    }
+    for (int i = ng; i < MAX_GROUP; ++i) {
+      p.map_k[i] = p.map_k[0];
+      p.map_v[i] = p.map_v[0];
+      p.dk_sum[i] = p.dk_sum[0];
+      p.dv_sum[i] = p.dv_sum[0];
+      p.window[i] = p.window[0];
+      p.ctas_per_pair[i] = p.ctas_per_pair[0];
+      p.first_slot[i + 1] = slots;
+      p.cta_begin[i + 1] = p.cta_begin[ng];
+    }
+    p.n_groups = ng;
     p.B = s->B;
     p.S = s->S;
     p.Hq = s->Hq;
@@ -756,19 +811,14 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     p.causal = causal;
     p.scale = sc;
     p.scale_log2 = sc * 1.4426950408889634f;
-    const int n_jt = (s->S + BT - 1) / BT, n_qt = (s->S + BQ2 - 1) / BQ2, n_pairs = s->Hkv * s->B;
-    p.window = std::min(n_qt, std::max(kMinWindow, (kStepsPerCta + n * (s->Hq / s->Hkv) - 1) / (n * (s->Hq / s->Hkv))));
-    p.ctas_per_pair = 0;
-    for (int w = 0; w * p.window < n_qt; ++w)
-      p.ctas_per_pair += causal ? std::min(n_jt, ((w + 1) * p.window * BQ2 + BT - 1) / BT) : n_jt;
-    const size_t kv_bytes = size_t(s->B) * s->S * s->Hkv * dh * 4;
     timing_before(KVP_KERNEL_ATTN_BWD_AUX, stream);
-    if (cudaMemsetAsync(acc_base, 0, size_t(n) * acc_bytes, stream) != cudaSuccess ||
-        cudaMemsetAsync(dk_sum[d], 0, kv_bytes, stream) != cudaSuccess ||
-        cudaMemsetAsync(dv_sum[d], 0, kv_bytes, stream) != cudaSuccess)
-      return KVP_ERR_CUDA;
+    if (cudaMemsetAsync(acc_base, 0, size_t(slots) * acc_bytes, stream) != cudaSuccess) return KVP_ERR_CUDA;
+    for (int i = 0; i < ng; ++i)
+      if (cudaMemsetAsync(p.dk_sum[i], 0, kv_bytes, stream) != cudaSuccess ||
+          cudaMemsetAsync(p.dv_sum[i], 0, kv_bytes, stream) != cudaSuccess)
+        return KVP_ERR_CUDA;
     timing_after(KVP_KERNEL_ATTN_BWD_AUX, stream);
-    dim3 grid(n_pairs * p.ctas_per_pair);
+    dim3 grid(p.cta_begin[ng]);
     timing_before(KVP_KERNEL_ATTN_BWD, stream);
     if (dh == 128)
       bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::TOTAL, stream>>>(p);
@@ -778,14 +828,14 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
     note_launch();
     if (cudaGetLastError() != cudaSuccess) return KVP_ERR_CUDA;
     timing_before(KVP_KERNEL_ATTN_BWD_AUX, stream);
-    for (int i = 0; i < n; ++i) {
+    for (int i = 0; i < slots; ++i) {
       const size_t threads = dq_acc_floats(s->B, s->S, s->Hq, dh) / 8;
       const int blocks = int(min(size_t(sm_count()) * 16, (threads + 255) / 256));
       if (dh == 128)
-        dq_convert_kernel<128><<<blocks, 256, 0, stream>>>(p.dq_acc[i], reinterpret_cast<__nv_bfloat16*>(dq[members[i]]),
+        dq_convert_kernel<128><<<blocks, 256, 0, stream>>>(p.dq_acc[i], reinterpret_cast<__nv_bfloat16*>(dq[slot_layer[i]]),
                                                            s->B, s->S, s->Hq, sc);
       else
-        dq_convert_kernel<64><<<blocks, 256, 0, stream>>>(p.dq_acc[i], reinterpret_cast<__nv_bfloat16*>(dq[members[i]]),
+        dq_convert_kernel<64><<<blocks, 256, 0, stream>>>(p.dq_acc[i], reinterpret_cast<__nv_bfloat16*>(dq[slot_layer[i]]),
                                                           s->B, s->S, s->Hq, sc);
       note_launch();
     }

@@ -20,6 +20,13 @@
  *  - dtype KVP_BF16: X, W, Q, K, V, O, dO, dQ, dX, Y are bf16 (round-to-nearest-even where
  *    the library stores them); LSE, dK/dV sums and all weight gradients are fp32; all
  *    accumulation is fp32.
+ *  - dtype KVP_F32 (the tiny-stack configuration's "fp32"): the same tensors are fp32 in the caller's memory.  The
+ *    library converts them on load to bf16 (round-to-nearest-even; values that are bf16-representable pass
+ *    unchanged) and widens its bf16 results on store, so the arithmetic, and the results, are those of KVP_BF16:
+ *    one code path.  The training entry points then keep the bf16 copies in the workspace (kvp_workspace_bytes
+ *    accounts for them, also for KVP_OP_PROJ_FWD / KVP_OP_ATTN_FWD, which need none otherwise); the decode entry
+ *    points read fp32 queries / new K, V rows and write fp32 outputs directly (the cache itself stays bf16).
+ *    kvp_out_proj_* and kvp_gemm take bf16 only.
  *  - Supported: dh in {64, 128}; Hq % Hkv == 0; D % 64 == 0; S >= 1.  Anything else returns
  *    KVP_ERR_UNSUPPORTED -- there is no slow path and no CPU fallback.
  *  - Kernels that wait on hardware barriers give up after about two seconds, record
@@ -47,7 +54,7 @@ enum {
   KVP_ERR_TIMEOUT = 6
 };
 
-enum { KVP_BF16 = 0 };
+enum { KVP_BF16 = 0, KVP_F32 = 1 };
 
 /* Returns a static string for a status code. */
 const char* kvp_status_string(int status);
@@ -157,7 +164,7 @@ int kvp_sim_1f1b(int32_t P, int32_t M, const int64_t* t_fwd, const int64_t* t_bw
  * ---------------------------------------------------------------------------------------- */
 typedef struct {
   int32_t L, B, S, D, Hq, Hkv, dh;
-  int32_t dtype; /* KVP_BF16 */
+  int32_t dtype; /* KVP_BF16 or KVP_F32 */
 } kvp_shape;
 
 enum { KVP_OP_PROJ_FWD = 0, KVP_OP_PROJ_BWD = 1, KVP_OP_ATTN_FWD = 2, KVP_OP_ATTN_BWD = 3, KVP_OP_DECODE = 4 };
@@ -240,7 +247,7 @@ typedef struct {
   int32_t max_pages;  /* columns of block_table */
   int32_t n_pages;    /* pages in each owner layer's pool */
   int32_t num_splits; /* KV splits per (sequence, KV head); 0 lets the library choose */
-  int32_t dtype;      /* KVP_BF16 */
+  int32_t dtype;      /* KVP_BF16, or KVP_F32: q, k_new, v_new, o are fp32; the cache is bf16 either way */
 } kvp_decode_desc;
 
 size_t kvp_decode_workspace_bytes(const kvp_decode_desc* d, const int32_t* donor);

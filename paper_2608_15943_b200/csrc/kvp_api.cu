@@ -1,5 +1,7 @@
 // C-ABI entry points of the training / prefill path: argument validation and the sequence of
 // kernel launches per layer.  No allocation, no synchronisation.
+#include <vector>
+
 #include "kvp_host.h"
 
 namespace kvp {
@@ -11,6 +13,7 @@ int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float sca
                  const float* const* lse, void* const* dq, float* const* dk_sum, float* const* dv_sum, void* ws,
                  size_t ws_bytes, cudaStream_t stream);
 int cast_f32_to_bf16(const float* src, void* dst, size_t n, cudaStream_t stream);
+int cast_bf16_to_f32(const void* src, float* dst, size_t n, cudaStream_t stream);
 
 namespace {
 
@@ -26,7 +29,7 @@ int check_donor(int L, const int32_t* donor) {
 int check_shape(const kvp_shape* s) {
   if (s == nullptr) return KVP_ERR_INVALID_ARG;
   if (s->L < 1 || s->B < 1 || s->S < 1 || s->D < 1 || s->Hq < 1 || s->Hkv < 1) return KVP_ERR_INVALID_ARG;
-  if (s->dtype != KVP_BF16) return KVP_ERR_UNSUPPORTED;
+  if (s->dtype != KVP_BF16 && s->dtype != KVP_F32) return KVP_ERR_UNSUPPORTED;
   if ((s->dh != 64 && s->dh != 128) || s->Hq % s->Hkv != 0 || s->D % 64 != 0) return KVP_ERR_UNSUPPORTED;
   return KVP_OK;
 }
@@ -42,13 +45,84 @@ bool ptrs_ok(const void* const* arr, int L, const int32_t* donor, bool owners_on
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
-}  // namespace
-}  // namespace kvp
+// ---------------------------------------------------------------------------------------------
+// KVP_F32 interface: bf16 shadow copies of the caller's fp32 tensors, carved from the workspace behind the
+// operation's own scratch.  Inputs are rounded on the way in, outputs widened on the way out; in between the
+// bf16 entry point runs unchanged.
+// ---------------------------------------------------------------------------------------------
+struct TensorSet {   // one per-layer tensor array of an entry point
+  size_t elems;      // elements per layer
+  bool owners_only;
+};
 
-using namespace kvp;
+size_t shadow_bytes(const kvp_shape* s, const int32_t* donor, const TensorSet* sets, int n_sets) {
+  size_t total = 0;
+  for (int i = 0; i < n_sets; ++i)
+    for (int l = 0; l < s->L; ++l)
+      if (!sets[i].owners_only || donor[l] == l) total += align256(sets[i].elems * 2);
+  return total;
+}
 
-extern "C" size_t kvp_workspace_bytes(int op, const kvp_shape* s, const int32_t* donor) {
-  if (check_shape(s) != KVP_OK || check_donor(s->L, donor) != KVP_OK) return 0;
+class Shadows {
+ public:
+  Shadows(const kvp_shape* s, const int32_t* donor, void* ws, size_t offset, cudaStream_t stream)
+      : s_(s), donor_(donor), cur_(reinterpret_cast<uint8_t*>(ws) + offset), stream_(stream) {}
+  // bf16 copies of an fp32 input array
+  const void* const* in(const void* const* src, const TensorSet& t) {
+    std::vector<void*>& arr = reserve(t);
+    for (int l = 0; l < s_->L; ++l)
+      if (arr[l] != nullptr && rc_ == KVP_OK) rc_ = cast_f32_to_bf16(reinterpret_cast<const float*>(src[l]), arr[l], t.elems, stream_);
+    return reinterpret_cast<const void* const*>(arr.data());
+  }
+  // bf16 buffers standing in for an fp32 output array; finish() widens them into the caller's tensors
+  void* const* out(void* const* dst, const TensorSet& t) {
+    std::vector<void*>& arr = reserve(t);
+    for (int l = 0; l < s_->L; ++l)
+      if (arr[l] != nullptr) pending_.push_back(Pending{arr[l], reinterpret_cast<float*>(dst[l]), t.elems});
+    return arr.data();
+  }
+  int status() const { return rc_; }
+  int finish() {
+    for (const Pending& p : pending_)
+      if (rc_ == KVP_OK) rc_ = cast_bf16_to_f32(p.src, p.dst, p.elems, stream_);
+    return rc_;
+  }
+
+ private:
+  struct Pending {
+    const void* src;
+    float* dst;
+    size_t elems;
+  };
+  std::vector<void*>& reserve(const TensorSet& t) {
+    arrays_.emplace_back(size_t(s_->L), nullptr);
+    std::vector<void*>& arr = arrays_.back();
+    for (int l = 0; l < s_->L; ++l)
+      if (!t.owners_only || donor_[l] == l) {
+        arr[l] = cur_;
+        cur_ += align256(t.elems * 2);
+      }
+    return arr;
+  }
+  const kvp_shape* s_;
+  const int32_t* donor_;
+  uint8_t* cur_;
+  cudaStream_t stream_;
+  int rc_ = KVP_OK;
+  std::vector<std::vector<void*>> arrays_;
+  std::vector<Pending> pending_;
+};
+
+struct Sizes {
+  TensorSet x, wq, wkv, q, kv;
+};
+Sizes sizes_of(const kvp_shape* s) {
+  const size_t T = size_t(s->B) * s->S, D = s->D, nq = size_t(s->Hq) * s->dh, nkv = size_t(s->Hkv) * s->dh;
+  return Sizes{{T * D, false}, {nq * D, false}, {nkv * D, true}, {T * nq, false}, {T * nkv, true}};
+}
+
+// scratch the bf16 form of an operation needs (before any shadows)
+size_t op_scratch_bytes(int op, const kvp_shape* s, const int32_t* donor) {
   switch (op) {
     case KVP_OP_PROJ_BWD:
       // bf16 copies of one owner's dk_sum and dv_sum
@@ -60,11 +134,44 @@ extern "C" size_t kvp_workspace_bytes(int op, const kvp_shape* s, const int32_t*
   }
 }
 
+size_t op_shadow_bytes(int op, const kvp_shape* s, const int32_t* donor) {
+  if (s->dtype != KVP_F32) return 0;
+  const Sizes z = sizes_of(s);
+  switch (op) {
+    case KVP_OP_PROJ_FWD: {
+      const TensorSet sets[] = {z.x, z.wq, z.wkv, z.wkv, z.q, z.kv, z.kv};
+      return shadow_bytes(s, donor, sets, 7);
+    }
+    case KVP_OP_PROJ_BWD: {
+      const TensorSet sets[] = {z.x, z.wq, z.wkv, z.wkv, z.q, z.x};   // x, wq, wk, wv, dq in; dx out
+      return shadow_bytes(s, donor, sets, 6);
+    }
+    case KVP_OP_ATTN_FWD: {
+      const TensorSet sets[] = {z.q, z.kv, z.kv, z.q};                // q, k, v in; o out
+      return shadow_bytes(s, donor, sets, 4);
+    }
+    case KVP_OP_ATTN_BWD: {
+      const TensorSet sets[] = {z.q, z.kv, z.kv, z.q, z.q, z.q};      // q, k, v, o, dO in; dq out
+      return shadow_bytes(s, donor, sets, 6);
+    }
+    default:
+      return 0;
+  }
+}
+
+}  // namespace
+}  // namespace kvp
+
+using namespace kvp;
+
+extern "C" size_t kvp_workspace_bytes(int op, const kvp_shape* s, const int32_t* donor) {
+  if (check_shape(s) != KVP_OK || check_donor(s->L, donor) != KVP_OK) return 0;
+  return align256(op_scratch_bytes(op, s, donor)) + op_shadow_bytes(op, s, donor);
+}
+
 extern "C" int kvp_proj_fwd(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
                             const void* const* wk, const void* const* wv, void* const* q, void* const* k,
                             void* const* v, void* ws, size_t ws_bytes, kvp_stream_t stream_) {
-  (void)ws;
-  (void)ws_bytes;
   int rc = check_shape(s);
   if (rc == KVP_OK) rc = check_donor(s->L, donor);
   if (rc != KVP_OK) return rc;
@@ -73,6 +180,23 @@ extern "C" int kvp_proj_fwd(const kvp_shape* s, const int32_t* donor, const void
       !ptrs_ok(v, s->L, donor, true))
     return KVP_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (s->dtype == KVP_F32) {
+    if (ws == nullptr || ws_bytes < kvp_workspace_bytes(KVP_OP_PROJ_FWD, s, donor) || !aligned16(ws)) return KVP_ERR_WORKSPACE;
+    const Sizes z = sizes_of(s);
+    Shadows sh(s, donor, ws, align256(op_scratch_bytes(KVP_OP_PROJ_FWD, s, donor)), stream);
+    const void* const* x16 = sh.in(x, z.x);
+    const void* const* wq16 = sh.in(wq, z.wq);
+    const void* const* wk16 = sh.in(wk, z.wkv);
+    const void* const* wv16 = sh.in(wv, z.wkv);
+    void* const* q16 = sh.out(q, z.q);
+    void* const* k16 = sh.out(k, z.kv);
+    void* const* v16 = sh.out(v, z.kv);
+    if (sh.status() != KVP_OK) return sh.status();
+    kvp_shape s16 = *s;
+    s16.dtype = KVP_BF16;
+    rc = kvp_proj_fwd(&s16, donor, x16, wq16, wk16, wv16, q16, k16, v16, ws, ws_bytes, stream_);
+    return rc != KVP_OK ? rc : sh.finish();
+  }
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh, Nkv = s->Hkv * s->dh;
   for (int l = 0; l < s->L; ++l) {
     GemmSeg sq{x[l], wq[l], D, D, D};
@@ -109,6 +233,21 @@ extern "C" int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void
   const size_t need = kvp_workspace_bytes(KVP_OP_PROJ_BWD, s, donor);
   if (ws == nullptr || ws_bytes < need || !aligned16(ws)) return KVP_ERR_WORKSPACE;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (s->dtype == KVP_F32) {
+    const Sizes z = sizes_of(s);
+    Shadows sh(s, donor, ws, align256(op_scratch_bytes(KVP_OP_PROJ_BWD, s, donor)), stream);
+    const void* const* x16 = sh.in(x, z.x);
+    const void* const* wq16 = sh.in(wq, z.wq);
+    const void* const* wk16 = sh.in(wk, z.wkv);
+    const void* const* wv16 = sh.in(wv, z.wkv);
+    const void* const* dq16 = sh.in(dq, z.q);
+    void* const* dx16 = sh.out(dx, z.x);
+    if (sh.status() != KVP_OK) return sh.status();
+    kvp_shape s16 = *s;
+    s16.dtype = KVP_BF16;
+    rc = kvp_proj_bwd(&s16, donor, x16, wq16, wk16, wv16, dq16, dk_sum, dv_sum, dwq, dwk, dwv, dx16, ws, ws_bytes, stream_);
+    return rc != KVP_OK ? rc : sh.finish();
+  }
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh, Nkv = s->Hkv * s->dh;
   const size_t n_kv = size_t(T) * Nkv;
   uint8_t* dk_bf = reinterpret_cast<uint8_t*>(ws);
@@ -144,6 +283,7 @@ extern "C" int kvp_out_proj_fwd(const kvp_shape* s, const void* const* o, const 
                                 kvp_stream_t stream_) {
   int rc = check_shape(s);
   if (rc != KVP_OK) return rc;
+  if (s->dtype != KVP_BF16) return KVP_ERR_UNSUPPORTED;
   if (o == nullptr || wo == nullptr || y == nullptr) return KVP_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh;
@@ -160,6 +300,7 @@ extern "C" int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const 
                                 const void* const* dy, void* const* d_o, float* const* dwo, kvp_stream_t stream_) {
   int rc = check_shape(s);
   if (rc != KVP_OK) return rc;
+  if (s->dtype != KVP_BF16) return KVP_ERR_UNSUPPORTED;
   if (o == nullptr || wo == nullptr || dy == nullptr || d_o == nullptr || dwo == nullptr) return KVP_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh;
@@ -181,8 +322,6 @@ extern "C" int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const 
 extern "C" int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
                             const void* const* k, const void* const* v, void* const* o, float* const* lse, void* ws,
                             size_t ws_bytes, kvp_stream_t stream_) {
-  (void)ws;
-  (void)ws_bytes;
   int rc = check_shape(s);
   if (rc == KVP_OK) rc = check_donor(s->L, donor);
   if (rc != KVP_OK) return rc;
@@ -191,6 +330,20 @@ extern "C" int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal
     return KVP_ERR_INVALID_ARG;
   if (scale < 0.f) return KVP_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (s->dtype == KVP_F32) {
+    if (ws == nullptr || ws_bytes < kvp_workspace_bytes(KVP_OP_ATTN_FWD, s, donor) || !aligned16(ws)) return KVP_ERR_WORKSPACE;
+    const Sizes z = sizes_of(s);
+    Shadows sh(s, donor, ws, align256(op_scratch_bytes(KVP_OP_ATTN_FWD, s, donor)), stream);
+    const void* const* q16 = sh.in(q, z.q);
+    const void* const* k16 = sh.in(k, z.kv);
+    const void* const* v16 = sh.in(v, z.kv);
+    void* const* o16 = sh.out(o, z.q);
+    if (sh.status() != KVP_OK) return sh.status();
+    kvp_shape s16 = *s;
+    s16.dtype = KVP_BF16;
+    rc = kvp_attn_fwd(&s16, donor, causal, scale, q16, k16, v16, o16, lse, ws, ws_bytes, stream_);
+    return rc != KVP_OK ? rc : sh.finish();
+  }
   for (int l = 0; l < s->L; ++l) {
     const int d = donor[l];
     rc = attn_fwd_layer(s, causal, scale, q[l], k[d], v[d], o[l], lse[l], stream);
@@ -213,8 +366,23 @@ extern "C" int kvp_attn_bwd(const kvp_shape* s, const int32_t* donor, int causal
       !ptrs_ok(reinterpret_cast<const void* const*>(dv_sum), s->L, donor, true))
     return KVP_ERR_INVALID_ARG;
   if (scale < 0.f) return KVP_ERR_INVALID_ARG;
-  const size_t need = attn_bwd_workspace(s, donor);
+  const size_t need = kvp_workspace_bytes(KVP_OP_ATTN_BWD, s, donor);
   if (need > 0 && (ws == nullptr || ws_bytes < need || !aligned16(ws))) return KVP_ERR_WORKSPACE;
+  if (s->dtype == KVP_F32) {
+    const Sizes z = sizes_of(s);
+    Shadows sh(s, donor, ws, align256(op_scratch_bytes(KVP_OP_ATTN_BWD, s, donor)), reinterpret_cast<cudaStream_t>(stream_));
+    const void* const* q16 = sh.in(q, z.q);
+    const void* const* k16 = sh.in(k, z.kv);
+    const void* const* v16 = sh.in(v, z.kv);
+    const void* const* o16 = sh.in(o, z.q);
+    const void* const* do16 = sh.in(d_o, z.q);
+    void* const* dq16 = sh.out(dq, z.q);
+    if (sh.status() != KVP_OK) return sh.status();
+    kvp_shape s16 = *s;
+    s16.dtype = KVP_BF16;
+    rc = kvp_attn_bwd(&s16, donor, causal, scale, q16, k16, v16, o16, do16, lse, dq16, dk_sum, dv_sum, ws, ws_bytes, stream_);
+    return rc != KVP_OK ? rc : sh.finish();
+  }
   return attn_bwd_all(s, donor, causal, scale, q, k, v, o, d_o, lse, dq, dk_sum, dv_sum, ws, ws_bytes,
                       reinterpret_cast<cudaStream_t>(stream_));
 }

@@ -32,8 +32,8 @@ __device__ int g_dec_status;
 struct DecGroup {
   const __nv_bfloat16* k_cache;
   const __nv_bfloat16* v_cache;
-  const __nv_bfloat16* q[MAX_MEMBERS];   // [B,Hq,dh]
-  __nv_bfloat16* o[MAX_MEMBERS];         // [B,Hq,dh]
+  const void* q[MAX_MEMBERS];            // [B,Hq,dh], bf16 or (io_f32) fp32
+  void* o[MAX_MEMBERS];                  // [B,Hq,dh], bf16 or (io_f32) fp32
   float* lse[MAX_MEMBERS];               // [B,Hq]
   int n_members;
   int pad;
@@ -46,6 +46,7 @@ struct DecParams {
   float* part_o;               // [n_groups][B][Hkv][NS][16][DH]
   float* part_ml;              // [n_groups][B][Hkv][NS][16][2]
   int B, Hq, Hkv, page_size, max_pages, n_pages, num_splits;
+  int io_f32;                  // queries are read and outputs written as fp32 (rounded to bf16 on load / widened on store)
   float scale_log2;
 };
 
@@ -127,17 +128,24 @@ __global__ void __launch_bounds__(DEC_THREADS, 2) decode_kernel(const __grid_con
   uint32_t qa[KSTEPS][4];
   {
     const int r0 = g, r1 = g + 8;
-    const __nv_bfloat16* q0 = nullptr;
-    const __nv_bfloat16* q1 = nullptr;
-    if (r0 < R) q0 = grp.q[r0 / G] + (size_t(b) * p.Hq + hk * G + r0 % G) * DH;
-    if (r1 < R) q1 = grp.q[r1 / G] + (size_t(b) * p.Hq + hk * G + r1 % G) * DH;
+    const size_t off0 = r0 < R ? (size_t(b) * p.Hq + hk * G + r0 % G) * DH : 0;
+    const size_t off1 = r1 < R ? (size_t(b) * p.Hq + hk * G + r1 % G) * DH : 0;
+    auto pair_at = [&](const void* base, size_t off, int c) -> uint32_t {   // elements c, c+1 of a query row as bf16
+      if (p.io_f32) {
+        const float2 f = *reinterpret_cast<const float2*>(reinterpret_cast<const float*>(base) + off + c);
+        return pack_bf16(f.x, f.y);
+      }
+      return *reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(base) + off + c);
+    };
+    const void* q0 = r0 < R ? grp.q[r0 / G] : nullptr;
+    const void* q1 = r1 < R ? grp.q[r1 / G] : nullptr;
 #pragma unroll
     for (int ks = 0; ks < KSTEPS; ++ks) {
       const int c = ks * 16 + t * 2;
-      qa[ks][0] = q0 ? *reinterpret_cast<const uint32_t*>(q0 + c) : 0u;
-      qa[ks][1] = q1 ? *reinterpret_cast<const uint32_t*>(q1 + c) : 0u;
-      qa[ks][2] = q0 ? *reinterpret_cast<const uint32_t*>(q0 + c + 8) : 0u;
-      qa[ks][3] = q1 ? *reinterpret_cast<const uint32_t*>(q1 + c + 8) : 0u;
+      qa[ks][0] = q0 ? pair_at(q0, off0, c) : 0u;
+      qa[ks][1] = q1 ? pair_at(q1, off1, c) : 0u;
+      qa[ks][2] = q0 ? pair_at(q0, off0, c + 8) : 0u;
+      qa[ks][3] = q1 ? pair_at(q1, off1, c + 8) : 0u;
     }
   }
 
@@ -343,20 +351,24 @@ __global__ void decode_combine_kernel(const __grid_constant__ DecParams p) {
       ll += f * p.part_ml[((unit0 + s) * 16 + row) * 2 + 1];
     }
     const int mem = row / G, hq = hk * G + row % G;
-    grp.o[mem][(size_t(b) * p.Hq + hq) * DH + col] = __float2bfloat16_rn(acc / ll);
+    const __nv_bfloat16 val = __float2bfloat16_rn(acc / ll);   // rounded to bf16 either way: one set of results
+    const size_t at = (size_t(b) * p.Hq + hq) * DH + col;
+    if (p.io_f32) reinterpret_cast<float*>(grp.o[mem])[at] = __bfloat162float(val);
+    else reinterpret_cast<__nv_bfloat16*>(grp.o[mem])[at] = val;
     if (col == 0) grp.lse[mem][size_t(b) * p.Hq + hq] = (mm + log2f(ll)) * 0.6931471805599453f;
   }
 }
 
 // Owners write the new token's K and V rows into their pages.
 struct AppendParams {
-  const __nv_bfloat16* k_new[MAX_DEC_GROUPS];
-  const __nv_bfloat16* v_new[MAX_DEC_GROUPS];
+  const void* k_new[MAX_DEC_GROUPS];   // [B,Hkv,dh] bf16, or fp32 when new_f32 (rounded to bf16 as it is stored)
+  const void* v_new[MAX_DEC_GROUPS];
   __nv_bfloat16* k_cache[MAX_DEC_GROUPS];
   __nv_bfloat16* v_cache[MAX_DEC_GROUPS];
   const int32_t* block_table;
   const int32_t* lengths;
   int B, Hkv, dh, page_size, max_pages, n_pages;
+  int new_f32;
 };
 
 __global__ void append_kernel(const __grid_constant__ AppendParams p) {
@@ -373,8 +385,16 @@ __global__ void append_kernel(const __grid_constant__ AppendParams p) {
     const int hk = idx / row_chunks, c = idx % row_chunks;
     const size_t src = (size_t(b) * p.Hkv + hk) * p.dh + c * 8;
     const size_t dst = ((size_t(page) * p.Hkv + hk) * p.page_size + pos % p.page_size) * p.dh + c * 8;
-    *reinterpret_cast<uint4*>(p.k_cache[layer] + dst) = *reinterpret_cast<const uint4*>(p.k_new[layer] + src);
-    *reinterpret_cast<uint4*>(p.v_cache[layer] + dst) = *reinterpret_cast<const uint4*>(p.v_new[layer] + src);
+    auto eight = [&](const void* base) -> uint4 {   // eight consecutive elements as bf16
+      if (p.new_f32) {
+        const float4 a = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(base) + src);
+        const float4 c4 = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(base) + src + 4);
+        return make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(c4.x, c4.y), pack_bf16(c4.z, c4.w));
+      }
+      return *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(base) + src);
+    };
+    *reinterpret_cast<uint4*>(p.k_cache[layer] + dst) = eight(p.k_new[layer]);
+    *reinterpret_cast<uint4*>(p.v_cache[layer] + dst) = eight(p.v_new[layer]);
   }
 }
 
@@ -382,7 +402,7 @@ int check_desc(const kvp_decode_desc* d) {
   if (d == nullptr) return KVP_ERR_INVALID_ARG;
   if (d->L < 1 || d->B < 1 || d->Hq < 1 || d->Hkv < 1 || d->max_pages < 1 || d->n_pages < 1 || d->num_splits < 0)
     return KVP_ERR_INVALID_ARG;
-  if (d->dtype != KVP_BF16) return KVP_ERR_UNSUPPORTED;
+  if (d->dtype != KVP_BF16 && d->dtype != KVP_F32) return KVP_ERR_UNSUPPORTED;
   if ((d->dh != 64 && d->dh != 128) || d->Hq % d->Hkv != 0 || d->Hq / d->Hkv > 16 || d->page_size < GRAN ||
       d->page_size % GRAN != 0)
     return KVP_ERR_UNSUPPORTED;
@@ -486,14 +506,15 @@ extern "C" int kvp_cache_append(const kvp_decode_desc* d, const int32_t* donor, 
   p.page_size = d->page_size;
   p.max_pages = d->max_pages;
   p.n_pages = d->n_pages;
+  p.new_f32 = d->dtype == KVP_F32;
   int n = 0;
   for (int l = 0; l <= d->L; ++l) {
     const bool owner = l < d->L && donor[l] == l;  // consumers store nothing (Eq. 3)
     if (owner) {
       if (k_new[l] == nullptr || v_new[l] == nullptr || k_cache[l] == nullptr || v_cache[l] == nullptr)
         return KVP_ERR_INVALID_ARG;
-      p.k_new[n] = reinterpret_cast<const __nv_bfloat16*>(k_new[l]);
-      p.v_new[n] = reinterpret_cast<const __nv_bfloat16*>(v_new[l]);
+      p.k_new[n] = k_new[l];
+      p.v_new[n] = v_new[l];
       p.k_cache[n] = reinterpret_cast<__nv_bfloat16*>(k_cache[l]);
       p.v_cache[n] = reinterpret_cast<__nv_bfloat16*>(v_cache[l]);
       ++n;
@@ -542,6 +563,7 @@ extern "C" int kvp_decode(const kvp_decode_desc* d, const int32_t* donor, float 
   p.max_pages = d->max_pages;
   p.n_pages = d->n_pages;
   p.num_splits = ns;
+  p.io_f32 = d->dtype == KVP_F32;
   const float sc = scale == 0.f ? 1.f / sqrtf(float(d->dh)) : scale;
   p.scale_log2 = sc * 1.4426950408889634f;
 
@@ -566,8 +588,8 @@ extern "C" int kvp_decode(const kvp_decode_desc* d, const int32_t* donor, float 
       for (int m = 0; m < MAX_MEMBERS; ++m) {
         const int l = sg.members[m < sg.n ? m : 0];
         if (q[l] == nullptr || o[l] == nullptr || lse[l] == nullptr) return KVP_ERR_INVALID_ARG;
-        g.q[m] = reinterpret_cast<const __nv_bfloat16*>(q[l]);
-        g.o[m] = reinterpret_cast<__nv_bfloat16*>(o[l]);
+        g.q[m] = q[l];
+        g.o[m] = o[l];
         g.lse[m] = lse[l];
       }
     }

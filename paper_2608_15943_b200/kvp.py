@@ -23,6 +23,7 @@ PLAN_STOP_ON_NO_IMPROVE, PLAN_STAGE_LOCAL_DONOR = 1, 2
 STOP_TOLERANCE, STOP_BUDGET, STOP_EXHAUSTED, STOP_NO_IMPROVE = range(4)
 PLACE_ARCH_BALANCED, PLACE_UNIFORM, PLACE_BIPOLAR = range(3)
 OP_PROJ_FWD, OP_PROJ_BWD, OP_ATTN_FWD, OP_ATTN_BWD, OP_DECODE = range(5)
+BF16, F32 = 0, 1   # dtype of the activations / weights in the caller's memory (kvp_shape.dtype, kvp_decode_desc.dtype)
 
 EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events",
            "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_sim_1f1b", "kvp_workspace_bytes",

@@ -396,6 +396,101 @@ def test_decode_ignores_never_appended_slots_even_if_they_hold_nan(kvp):
     assert kvp.device_status() == kvp.OK
 
 
+def test_c0_with_fp32_buffers(kvp):
+    """The tiny stack with fp32 tensors in the caller's memory (dtype F32): forward, backward and decode steps.
+    The library rounds fp32 inputs to bf16 on load and widens its bf16 results on store, so (i) every output
+    meets the oracle at the bf16 tolerances and (ii) equals, bit for bit after widening, what the bf16 interface
+    returns for the same values (the generator's values are bf16-representable)."""
+    cfg = W.C0
+    t = W.make_train_inputs(cfg, "cuda")
+    out = W.alloc_train_outputs(cfg, "cuda")
+    run_block(kvp, cfg, t, out)                                   # bf16 interface: the comparison values
+    f32 = lambda xs: [None if a is None else a.float() for a in xs]
+    t32 = {n: f32(xs) for n, xs in t.items()}
+    like = lambda xs: [None if a is None else torch.full(a.shape, float("nan"), device="cuda") for a in xs]
+    o32 = {n: like(out[n]) for n in ("q", "k", "v", "o", "dq", "dx")}
+    lse = like(out["lse"])
+    dk, dv, dwq, dwk, dwv = (like(out[n]) for n in ("dk_sum", "dv_sum", "dwq", "dwk", "dwv"))
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh, kvp.F32)
+    need = max(kvp.workspace_bytes(op, sh, cfg.donor) for op in (kvp.OP_PROJ_FWD, kvp.OP_ATTN_FWD, kvp.OP_ATTN_BWD, kvp.OP_PROJ_BWD))
+    assert kvp.workspace_bytes(kvp.OP_PROJ_FWD, sh, cfg.donor) > 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    with pytest.raises(kvp.KvpError) as e:                        # the fp32 interface needs its shadow space
+        kvp.proj_fwd(sh, cfg.donor, t32["x"], t32["wq"], t32["wk"], t32["wv"], o32["q"], o32["k"], o32["v"])
+    assert e.value.status == kvp.ERR_WORKSPACE
+    kvp.proj_fwd(sh, cfg.donor, t32["x"], t32["wq"], t32["wk"], t32["wv"], o32["q"], o32["k"], o32["v"], ws)
+    kvp.attn_fwd(sh, cfg.donor, o32["q"], o32["k"], o32["v"], o32["o"], lse, ws=ws)
+    kvp.attn_bwd(sh, cfg.donor, o32["q"], o32["k"], o32["v"], o32["o"], t32["d_o"], lse, o32["dq"], dk, dv, ws)
+    kvp.proj_bwd(sh, cfg.donor, t32["x"], t32["wq"], t32["wk"], t32["wv"], o32["dq"], dk, dv, dwq, dwk, dwv, o32["dx"], ws)
+    torch.cuda.synchronize()
+    assert kvp.device_status() == kvp.OK
+    for n in ("q", "k", "v", "o", "dx"):
+        for l in range(cfg.L):
+            if out[n][l] is not None:
+                assert o32[n][l].dtype == torch.float32
+                assert torch.equal(o32[n][l], out[n][l].float()), (n, l)
+    for l in range(cfg.L):
+        assert torch.equal(lse[l], out["lse"][l])
+        # dQ goes through fp32 reductions whose order is not fixed: equal up to fp32 rounding, then bf16-rounded
+        assert (o32["dq"][l] - out["dq"][l].float()).abs().max().item() <= 2.0 ** -7 * out["dq"][l].float().abs().max().item()
+    # against the oracle, per operation, on the operands each operation consumed
+    dims = (cfg.B, cfg.S, cfg.Hq, cfg.Hkv, cfg.dh)
+    x, wq, wk, wv, d_o = (f64l(t[n]) for n in ("x", "wq", "wk", "wv", "d_o"))
+    q, k, v = A.proj_fwd(x, wq, wk, wv, cfg.donor, *dims)
+    qs, ks, vs = f64l(o32["q"]), f64l(o32["k"]), f64l(o32["v"])
+    ro, rl = A.attn_fwd(qs, ks, vs, cfg.donor)
+    rdq, rdk, rdv = A.attn_bwd(qs, ks, vs, d_o, cfg.donor)
+    for l in range(cfg.L):
+        close(f"q[{l}]", o32["q"][l], q[l])
+        close(f"o[{l}]", o32["o"][l], ro[l])
+        lse_close(f"lse[{l}]", lse[l], rl[l])
+        close(f"dq[{l}]", o32["dq"][l], rdq[l])
+        if cfg.donor[l] == l:
+            close(f"dk_sum[{l}]", dk[l], rdk[l], sum_over_tokens=True)
+            close(f"dv_sum[{l}]", dv[l], rdv[l], sum_over_tokens=True)
+    # decode with fp32 queries / new rows / outputs over a bf16 cache filled from the prefill
+    steps, page = 4, 16
+    own = cfg.owners()
+    max_pages = (cfg.S + steps + page - 1) // page
+    n_pages = cfg.B * max_pages
+    bt = torch.arange(n_pages, dtype=torch.int32, device="cuda").reshape(cfg.B, max_pages)
+    kc, vc, kc16, vc16 = ([None] * cfg.L for _ in range(4))
+    for l in own:
+        for name, pools in (("k", (kc, kc16)), ("v", (vc, vc16))):
+            pool = torch.zeros(n_pages, cfg.Hkv, page, cfg.dh, dtype=torch.bfloat16, device="cuda")
+            pg = out[name][l].reshape(cfg.B, cfg.S // page, page, cfg.Hkv, cfg.dh).permute(0, 1, 3, 2, 4)
+            pool.view(cfg.B, max_pages, cfg.Hkv, page, cfg.dh)[:, :cfg.S // page] = pg
+            pools[0][l], pools[1][l] = pool, pool.clone()
+    d32 = kvp.DecodeDesc(cfg.L, cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, page, max_pages, n_pages, 2, kvp.F32)
+    d16 = kvp.DecodeDesc(cfg.L, cfg.B, cfg.Hq, cfg.Hkv, cfg.dh, page, max_pages, n_pages, 2)
+    dws = torch.empty(kvp.decode_workspace_bytes(d32, cfg.donor), dtype=torch.uint8, device="cuda")
+    lengths = torch.full((cfg.B,), cfg.S, dtype=torch.int32, device="cuda")
+    for step in range(steps):
+        qn = [synth.normal((cfg.B, cfg.Hq, cfg.dh), W.SEED, synth.tid(30, l, step), 1.0, "cuda") for l in range(cfg.L)]
+        kn = [synth.normal((cfg.B, cfg.Hkv, cfg.dh), W.SEED, synth.tid(31, l, step), 1.0, "cuda") if l in own else None
+              for l in range(cfg.L)]
+        vn = [synth.normal((cfg.B, cfg.Hkv, cfg.dh), W.SEED, synth.tid(32, l, step), 1.0, "cuda") if l in own else None
+              for l in range(cfg.L)]
+        lengths += 1
+        kvp.cache_append(d32, cfg.donor, f32(kn), f32(vn), kc, vc, bt, lengths)
+        kvp.cache_append(d16, cfg.donor, kn, vn, kc16, vc16, bt, lengths)
+        o_a = [torch.full((cfg.B, cfg.Hq, cfg.dh), float("nan"), device="cuda") for _ in range(cfg.L)]
+        o_b = [torch.empty(cfg.B, cfg.Hq, cfg.dh, dtype=torch.bfloat16, device="cuda") for _ in range(cfg.L)]
+        l_a = [torch.empty(cfg.B, cfg.Hq, device="cuda") for _ in range(cfg.L)]
+        l_b = [torch.empty(cfg.B, cfg.Hq, device="cuda") for _ in range(cfg.L)]
+        kvp.decode(d32, cfg.donor, f32(qn), kc, vc, bt, lengths, o_a, l_a, dws)
+        kvp.decode(d16, cfg.donor, qn, kc16, vc16, bt, lengths, o_b, l_b, dws)
+        lens = [int(n) for n in lengths.cpu()]
+        ro, rl = decode_reference(qn, kc, vc, bt, lens, cfg.donor, page)
+        for l in range(cfg.L):
+            assert torch.equal(o_a[l], o_b[l].float()) and torch.equal(l_a[l], l_b[l])
+            close(f"decode step {step} o[{l}]", o_a[l], ro[l])
+            lse_close(f"decode step {step} lse[{l}]", l_a[l], rl[l])
+    for l in own:
+        assert torch.equal(kc[l], kc16[l]) and torch.equal(vc[l], vc16[l])
+    assert kvp.device_status() == kvp.OK
+
+
 def test_c0_prefill_then_16_decode_steps(kvp):
     """Prefill the tiny stack, move K/V into pages, then 16 decode steps: project the new token,
     append for owners, attend over the shared cache; compared step by step with the oracle run with

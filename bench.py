@@ -132,15 +132,20 @@ class TrainRunner:
         self.sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
         nq, nkv = cfg.Hq * cfg.dh, cfg.Hkv * cfg.dh
         own = set(cfg.owners())
-        if backward and bucket:   # weight gradients live in one flat bucket (one all-reduce per step for N > 1)
+        if backward and bucket:   # weight gradients live in one flat bucket, each layer's entries next to each other
             shapes = [(nq, cfg.D)] * cfg.L + [(nkv, cfg.D) if l in own else None for l in range(cfg.L)] * 2
+            layer_of = list(range(cfg.L)) * 3
             if out_proj:
                 shapes += [(cfg.D, nq)] * cfg.L
-            self.bucket = kdist.GradBucket(shapes, device)
+                layer_of += list(range(cfg.L))
+            self.bucket = kdist.GradBucket(shapes, device, layer_of=layer_of)
             v = self.bucket.views
             self.out["dwq"], self.out["dwk"], self.out["dwv"] = v[:cfg.L], v[cfg.L:2 * cfg.L], v[2 * cfg.L:3 * cfg.L]
             if out_proj:
                 self.out["dwo"] = v[3 * cfg.L:4 * cfg.L]
+            if kdist.is_multi():   # the cross-rank sum runs layer by layer on its own stream, behind the gradient GEMMs
+                self.s_comm = torch.cuda.Stream()
+                self.ev_layer = [torch.cuda.Event() for _ in range(cfg.L)]
         else:
             self.bucket = None
         ws = max(kvp.workspace_bytes(kvp.OP_ATTN_BWD, self.sh, cfg.donor),
@@ -165,10 +170,21 @@ class TrainRunner:
                    o["dv_sum"], self.ws)
         if before_proj_bwd is not None:
             before_proj_bwd()
-        k.proj_bwd(self.sh, c.donor, t["x"], t["wq"], t["wk"], t["wv"], o["dq"], o["dk_sum"], o["dv_sum"],
-                   o["dwq"], o["dwk"], o["dwv"], o["dx"], self.ws)
-        if self.bucket is not None:
-            self.bucket.all_reduce()
+        args = (self.sh, c.donor, t["x"], t["wq"], t["wk"], t["wv"], o["dq"], o["dk_sum"], o["dv_sum"], o["dwq"], o["dwk"],
+                o["dwv"], o["dx"], self.ws)
+        if self.bucket is not None and kdist.is_multi():
+            # one layer's gradient GEMMs, then that layer's slice of the bucket is summed over ranks on the side
+            # stream while the next layer's GEMMs run: only the last layer's reduction is exposed
+            cur = torch.cuda.current_stream()
+            for l in range(c.L):
+                k.proj_bwd(*args, layer_begin=l, layer_end=l + 1)
+                self.ev_layer[l].record(cur)
+                with torch.cuda.stream(self.s_comm):
+                    self.s_comm.wait_event(self.ev_layer[l])
+                    self.bucket.all_reduce_layer(l)
+            cur.wait_stream(self.s_comm)
+        else:
+            k.proj_bwd(*args)
 
     def flops(self):
         c = self.cfg

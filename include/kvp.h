@@ -189,6 +189,14 @@ int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void* const* x,
                  const float* const* dv_sum, float* const* dwq, float* const* dwk, float* const* dwv,
                  void* const* dx, void* ws, size_t ws_bytes, kvp_stream_t stream);
 
+/* kvp_proj_bwd restricted to layers layer_begin <= l < layer_end (same arrays of length L, same workspace): lets a
+ * data-parallel caller start the cross-rank sum of one layer's weight gradients while the next layer's are still
+ * being computed.  KVP_BF16 only. */
+int kvp_proj_bwd_range(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
+                       const void* const* wk, const void* const* wv, const void* const* dq, const float* const* dk_sum,
+                       const float* const* dv_sum, float* const* dwq, float* const* dwk, float* const* dwv,
+                       void* const* dx, int layer_begin, int layer_end, void* ws, size_t ws_bytes, kvp_stream_t stream);
+
 /* Output projection y[l] = o[l] wo[l]^T and its chain rule (d_o = dy wo, dwo = dy^T o); the paper's
  * 2bsh^2 "output projection" term.  o[l]: [B*S, Hq*dh]; wo[l]: [D, Hq*dh]; y[l]: [B*S, D]. */
 int kvp_out_proj_fwd(const kvp_shape* s, const void* const* o, const void* const* wo, void* const* y,

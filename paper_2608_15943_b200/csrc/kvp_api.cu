@@ -219,9 +219,19 @@ extern "C" int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void
                             const float* const* dk_sum, const float* const* dv_sum, float* const* dwq,
                             float* const* dwk, float* const* dwv, void* const* dx, void* ws, size_t ws_bytes,
                             kvp_stream_t stream_) {
+  return kvp_proj_bwd_range(s, donor, x, wq, wk, wv, dq, dk_sum, dv_sum, dwq, dwk, dwv, dx, 0, s != nullptr ? s->L : 0, ws,
+                            ws_bytes, stream_);
+}
+
+extern "C" int kvp_proj_bwd_range(const kvp_shape* s, const int32_t* donor, const void* const* x,
+                                  const void* const* wq, const void* const* wk, const void* const* wv,
+                                  const void* const* dq, const float* const* dk_sum, const float* const* dv_sum,
+                                  float* const* dwq, float* const* dwk, float* const* dwv, void* const* dx,
+                                  int layer_begin, int layer_end, void* ws, size_t ws_bytes, kvp_stream_t stream_) {
   int rc = check_shape(s);
   if (rc == KVP_OK) rc = check_donor(s->L, donor);
   if (rc != KVP_OK) return rc;
+  if (layer_begin < 0 || layer_end > s->L || layer_begin > layer_end) return KVP_ERR_INVALID_ARG;
   if (!ptrs_ok(x, s->L, donor, false) || !ptrs_ok(wq, s->L, donor, false) || !ptrs_ok(wk, s->L, donor, true) ||
       !ptrs_ok(wv, s->L, donor, true) || !ptrs_ok(dq, s->L, donor, false) ||
       !ptrs_ok(reinterpret_cast<const void* const*>(dk_sum), s->L, donor, true) ||
@@ -245,6 +255,7 @@ extern "C" int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void
     if (sh.status() != KVP_OK) return sh.status();
     kvp_shape s16 = *s;
     s16.dtype = KVP_BF16;
+    if (layer_begin != 0 || layer_end != s->L) return KVP_ERR_UNSUPPORTED;   // the fp32 interface converts whole arrays
     rc = kvp_proj_bwd(&s16, donor, x16, wq16, wk16, wv16, dq16, dk_sum, dv_sum, dwq, dwk, dwv, dx16, ws, ws_bytes, stream_);
     return rc != KVP_OK ? rc : sh.finish();
   }
@@ -252,7 +263,7 @@ extern "C" int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void
   const size_t n_kv = size_t(T) * Nkv;
   uint8_t* dk_bf = reinterpret_cast<uint8_t*>(ws);
   uint8_t* dv_bf = dk_bf + align256(n_kv * 2);
-  for (int l = 0; l < s->L; ++l) {
+  for (int l = layer_begin; l < layer_end; ++l) {
     // dWq = dQ^T X : A = dQ stored [T, Nq] (MN-major for M = Nq), B = X stored [T, D] (MN-major for N = D)
     GemmSeg swq{dq[l], x[l], Nq, D, T};
     rc = gemm_bf16(Nq, D, &swq, 1, 1, 1, dwq[l], D, 1, stream);

@@ -27,7 +27,7 @@ BF16, F32 = 0, 1   # dtype of the activations / weights in the caller's memory (
 
 EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events",
            "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_sim_1f1b", "kvp_workspace_bytes",
-           "kvp_proj_fwd", "kvp_proj_bwd", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
+           "kvp_proj_fwd", "kvp_proj_bwd", "kvp_proj_bwd_range", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
            "kvp_gemm", "kvp_rmsnorm", "kvp_rope", "kvp_swiglu", "kvp_add", "kvp_decode_workspace_bytes", "kvp_cache_append",
            "kvp_decode", "kvp_decode_static", "kvp_selftest_bounded_wait"]
 
@@ -233,6 +233,9 @@ lib.kvp_proj_fwd.restype = C.c_int
 lib.kvp_proj_fwd.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32)] + [_PP] * 7 + [C.c_void_p, C.c_size_t, C.c_void_p]
 lib.kvp_proj_bwd.restype = C.c_int
 lib.kvp_proj_bwd.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32)] + [_PP] * 11 + [C.c_void_p, C.c_size_t, C.c_void_p]
+lib.kvp_proj_bwd_range.restype = C.c_int
+lib.kvp_proj_bwd_range.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32)] + [_PP] * 11 + [C.c_int, C.c_int, C.c_void_p, C.c_size_t,
+                                                                                          C.c_void_p]
 lib.kvp_out_proj_fwd.restype = C.c_int
 lib.kvp_out_proj_fwd.argtypes = [C.POINTER(Shape)] + [_PP] * 3 + [C.c_void_p]
 lib.kvp_out_proj_bwd.restype = C.c_int
@@ -260,11 +263,17 @@ def proj_fwd(shape, donor, x, wq, wk, wv, q, k, v, ws=None):
            "kvp_proj_fwd")
 
 
-def proj_bwd(shape, donor, x, wq, wk, wv, dq, dk_sum, dv_sum, dwq, dwk, dwv, dx, ws):
+def proj_bwd(shape, donor, x, wq, wk, wv, dq, dk_sum, dv_sum, dwq, dwk, dwv, dx, ws, layer_begin=None, layer_end=None):
+    """kvp_proj_bwd, or kvp_proj_bwd_range when a layer range is given."""
     p, n = _ws(ws)
-    _check(lib.kvp_proj_bwd(C.byref(shape), _i32_array(donor), _ptr_array(x), _ptr_array(wq), _ptr_array(wk),
-                            _ptr_array(wv), _ptr_array(dq), _ptr_array(dk_sum), _ptr_array(dv_sum), _ptr_array(dwq),
-                            _ptr_array(dwk), _ptr_array(dwv), _ptr_array(dx), p, n, _stream()), "kvp_proj_bwd")
+    args = (C.byref(shape), _i32_array(donor), _ptr_array(x), _ptr_array(wq), _ptr_array(wk), _ptr_array(wv),
+            _ptr_array(dq), _ptr_array(dk_sum), _ptr_array(dv_sum), _ptr_array(dwq), _ptr_array(dwk), _ptr_array(dwv),
+            _ptr_array(dx))
+    if layer_begin is None and layer_end is None:
+        _check(lib.kvp_proj_bwd(*args, p, n, _stream()), "kvp_proj_bwd")
+    else:
+        _check(lib.kvp_proj_bwd_range(*args, int(layer_begin or 0), shape.L if layer_end is None else int(layer_end), p, n,
+                                      _stream()), "kvp_proj_bwd_range")
 
 
 def out_proj_fwd(shape, o, wo, y):

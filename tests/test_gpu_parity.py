@@ -396,6 +396,30 @@ def test_decode_ignores_never_appended_slots_even_if_they_hold_nan(kvp):
     assert kvp.device_status() == kvp.OK
 
 
+def test_projection_backward_layer_by_layer_equals_one_call(kvp):
+    """kvp_proj_bwd_range over single layers (what a data-parallel step interleaves with the per-layer gradient
+    all-reduce) writes bit for bit what one kvp_proj_bwd call writes."""
+    cfg = W.C0
+    t = W.make_train_inputs(cfg, "cuda")
+    out = W.alloc_train_outputs(cfg, "cuda")
+    sh = run_block(kvp, cfg, t, out)
+    ws = torch.empty(kvp.workspace_bytes(kvp.OP_PROJ_BWD, sh, cfg.donor), dtype=torch.uint8, device="cuda")
+    names = ("dwq", "dwk", "dwv", "dx")
+    again = {n: [None if a is None else torch.full_like(a, float("nan")) for a in out[n]] for n in names}
+    for l in range(cfg.L):
+        kvp.proj_bwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["dq"], out["dk_sum"], out["dv_sum"],
+                     again["dwq"], again["dwk"], again["dwv"], again["dx"], ws, layer_begin=l, layer_end=l + 1)
+    torch.cuda.synchronize()
+    for n in names:
+        for l in range(cfg.L):
+            if out[n][l] is not None:
+                assert torch.equal(again[n][l], out[n][l]), (n, l)
+    with pytest.raises(kvp.KvpError):
+        kvp.proj_bwd(sh, cfg.donor, t["x"], t["wq"], t["wk"], t["wv"], out["dq"], out["dk_sum"], out["dv_sum"],
+                     again["dwq"], again["dwk"], again["dwv"], again["dx"], ws, layer_begin=3, layer_end=9)
+    assert kvp.device_status() == kvp.OK
+
+
 def test_c0_with_fp32_buffers(kvp):
     """The tiny stack with fp32 tensors in the caller's memory (dtype F32): forward, backward and decode steps.
     The library rounds fp32 inputs to bf16 on load and widens its bf16 results on store, so (i) every output

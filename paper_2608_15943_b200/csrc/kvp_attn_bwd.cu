@@ -71,7 +71,7 @@ struct BwdSmem {
   static constexpr int OFF_ONES = OFF_DQ + 4 * DQ_STAGE_BYTES;     // [128 x 8] bf16: columns 0-7 of the tile of ones
   static constexpr int OFF_STAT = OFF_ONES + 2048;                 // [4 steps][lse, delta][64 x 8] bf16: columns 0-7
   static constexpr int OFF_ZERO = OFF_STAT + 8 * 1024;             // [128 x 8] zeros: columns 8-15 of all of the above
-  static constexpr int OFF_RAW = OFF_ZERO + 2048;                  // [4 statistics warps][8 steps][32] fp32 as loaded
+  static constexpr int OFF_RAW = OFF_ZERO + 2048;                  // [8 steps][lse, delta][64] fp32 as loaded
   static constexpr int OFF_BAR = OFF_RAW + 4096;
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;
 };
@@ -149,8 +149,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
   uint64_t* dp_free = st_full + 1;                // dP^T of the step is in registers (256 arrivals)
   uint64_t* pds_ready = dp_free + 1;              // [2] P^T, dS^T written (TMEM and shared memory), next statistics staged
   uint64_t* dq_full = pds_ready + 2;              // dQ^T of the step is in TMEM; its dS^T tile may be overwritten
-  uint64_t* dq_free = dq_full + 1;                // dQ^T of the step is in registers (128 arrivals)
-  uint64_t* stat0 = dq_free + 1;                  // statistics of the first steps staged (256 arrivals)
+  uint64_t* dq_free = dq_full + 1;                // dQ^T of the step is in registers, statistics of step +3 staged (128 arrivals)
+  uint64_t* stat0 = dq_free + 1;                  // statistics of the first steps staged (128 arrivals)
   uint64_t* acc_done = stat0 + 1;                 // all MMAs have completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
 
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
     for (int i = 0; i < 2; ++i) mbar_init(&pds_ready[i], 256);
     mbar_init(dq_full, 1);
     mbar_init(dq_free, 128);
-    mbar_init(stat0, 256);
+    mbar_init(stat0, 128);
     mbar_init(acc_done, 1);
     mbar_fence_init();
   }
@@ -349,81 +349,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
     const int r = quarter * 32 + lane;  // key row inside the tile == TMEM lane
     const uint32_t lane_sel = uint32_t(quarter * 32) << 16;
     const int kv_row = kv0 + r;
-    const float inv_scale = 1.f / p.scale;
-    // Statistics: in each warpgroup, lane quarter 0 stages -LSE/scale and quarter 1 stages -Delta of the
-    // warpgroup's 32 query columns as the three-term bf16 split the tensor core adds.  The raw fp32 values come
-    // in through cp.async into a small ring in shared memory, issued eight steps before the step that uses them
-    // and read back (and staged as an operand tile) three steps before: no register ever waits on global memory.
-    const int stat_kind = quarter ^ 2;  // 0 lse, 1 delta, others idle: the warps whose scheduler hosts no TMA / MMA warp
-    const bool stat_warp = stat_kind < 2;
-    uint8_t* stat_row = smem + L::OFF_STAT + (stat_kind & 1) * 1024 + (wg * 32 + lane) * 16;
-    float* raw = reinterpret_cast<float*>(smem + L::OFF_RAW) + ((wg * 2 + (stat_kind & 1)) * 8) * 32 + lane;
-    const float stat_mul = stat_kind == 0 ? -inv_scale : -1.f;
-    const float stat_pad = stat_kind == 0 ? -30000.f : 0.f;  // a query beyond the sequence: exp2 underflows to zero
-    // Two cursors walk the steps in order (incremental decode of step -> layer, head, query tile): one
-    // for the step whose statistics are requested next, one kStatAhead steps further that only pulls the
-    // line into L2.
-    constexpr int kStatAhead = 12;
-    // `row` is the statistic row of the cursor's (layer, head): it is looked up (an indexed read of the kernel
-    // parameters) only when the stream changes, never on the per-step path
-    struct Cursor {
-      int it = 0, qi = 0, g = 0, li = 0;
-      const float* row = nullptr;
-    };
-    auto row_of = [&](int li, int g) {
-      const int slot = slot0 + (li < n_layers ? li : 0);
-      const float* src = stat_kind == 0 ? p.lse[slot] : p.delta[slot];
-      return src + (size_t(b) * p.Hq + hk * G + g) * p.S;
-    };
-    auto advance = [&](Cursor& c) {
-      ++c.it;
-      if (++c.qi == per_stream) {
-        c.qi = 0;
-        if (++c.g == G) {
-          c.g = 0;
-          ++c.li;
-        }
-        c.row = row_of(c.li, c.g);
-      }
-    };
-    auto locate = [&](const Cursor& c, bool& valid) {  // address of this lane's statistic of step c (clamped, always valid)
-      const int qc = (qt_first + c.qi) * BQ2 + wg * 32 + lane;
-      valid = stat_warp && c.it < n_iter && qc < p.S;
-      return c.row + (valid ? qc : p.S - 1);
-    };
-    Cursor cf, cp;
-    cf.row = cp.row = row_of(0, 0);
-    for (int i = 0; i < kStatAhead; ++i) advance(cp);
-    auto request = [&]() -> bool {  // cp.async of the next step's value into its ring slot; returns its validity
-      bool ahead_valid, valid;
-      const float* ahead = locate(cp, ahead_valid);
-      if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(ahead));
-      advance(cp);
-      const float* ptr = locate(cf, valid);
-      if (stat_warp)
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(raw + (cf.it & 7) * 32)), "l"(ptr) : "memory");
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      advance(cf);
-      return valid;
-    };
-    auto stage = [&](int step, bool valid) {  // the value of `step` has landed: split it into the step's operand tile
-      if (stat_warp)
-        *reinterpret_cast<uint4*>(stat_row + (step & 3) * 2048) = split3_bf16(valid ? raw[(step & 7) * 32] * stat_mul : stat_pad);
-    };
-    // validity flags of the requests in flight, oldest (step it+3) in bit 0
-    uint32_t vbits = 0;
-    {
-      const bool a0 = request(), a1 = request(), a2 = request();
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-      stage(0, a0);
-      stage(1, a1);
-      stage(2, a2);
-      // steps 3..7; from here on a ring slot is requested again only after its previous value has been staged
-#pragma unroll
-      for (int i = 0; i < 5; ++i) vbits |= uint32_t(request()) << i;
-    }
-    fence_proxy_async_smem();
-    mbar_arrive(stat0);
     const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
     // P^T and dS^T (bf16 pairs) overwrite the warpgroup's OWN score columns, which the other warpgroup never
     // reads: P^T in 32-bit columns [wg*32, wg*32+16), dS^T in [wg*32+16, wg*32+32)
@@ -440,7 +365,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
       uint32_t st[32], dp[32];
       tmem_ld_x32(tm + lane_sel + col, st);
       tmem_ld_x32(tm_dp + lane_sel + col, dp);
-      vbits |= uint32_t(request()) << 5;  // statistics of step it+8
       const int q_col0 = (qt_first + qi) * BQ2 + wg * 32;           // query of this warpgroup's first column
       const bool diag = p.causal && q_col0 - wg * 32 < kv0 + BT;    // the query tile straddles the diagonal
       const int first_visible = diag ? kv_row - q_col0 : 0;         // own columns below this are masked for this key row
@@ -474,14 +398,9 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
         *reinterpret_cast<uint4*>(ds_smem + sw128_offset(r, wg * 4 + j)) =
             make_uint4(dk[4 * j], dk[4 * j + 1], dk[4 * j + 2], dk[4 * j + 3]);
       tmem_st_wait();
-      fence_proxy_async_smem();  // dS^T, and the statistics staged one step ago, are read by the tensor core's proxy
+      fence_proxy_async_smem();  // dS^T is read by the tensor core's proxy
       tc_fence_before_sync();
       mbar_arrive(&pds_ready[set]);
-      // Off the critical path: the tile of step it+3 (last read by the scores of step it-1, which have
-      // completed).  The next step's arrive publishes it, before the scores of step it+3 are issued.
-      asm volatile("cp.async.wait_group 5;" ::: "memory");
-      stage(it + 3, vbits & 1u);
-      vbits >>= 1;
       if (++qi == per_stream) qi = 0;
     }
     ok = __all_sync(0xffffffffu, ok);
@@ -522,6 +441,79 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
     const bool active = quarter * 32 < DH;  // with DH == 64 the upper lanes hold nothing
     float* stg = reinterpret_cast<float*>(smem + L::OFF_DQ + (warp - 10) * DQ_STAGE_BYTES);
     const uint32_t stg_s = smem_u32(stg);
+    // Statistics.  This warpgroup also prepares the per-query operand tiles the tensor core adds to the scores:
+    // thread t < 64 handles -LSE/scale of query column t, thread 64 + t handles -Delta of column t, as the
+    // three-term bf16 split.  The raw fp32 values come in through cp.async into a small ring in shared memory,
+    // requested eight steps before the step that uses them and staged as an operand tile three steps before: no
+    // register ever waits on global memory, and the compute warpgroups never touch the statistics.
+    const int stat_tid = threadIdx.x - 10 * 32;
+    const int stat_kind = stat_tid >> 6;   // 0 lse, 1 delta
+    const int stat_col = stat_tid & 63;
+    uint8_t* stat_row = smem + L::OFF_STAT + stat_kind * 1024 + stat_col * 16;
+    float* raw = reinterpret_cast<float*>(smem + L::OFF_RAW) + stat_tid;   // ring slot s at raw[s * 128]
+    const float stat_mul = stat_kind == 0 ? -1.f / p.scale : -1.f;
+    const float stat_pad = stat_kind == 0 ? -30000.f : 0.f;  // a query beyond the sequence: exp2 underflows to zero
+    // Two cursors walk the steps in order (incremental decode of step -> layer, head, query tile): one for the
+    // step whose statistics are requested next, one kStatAhead steps further that only pulls the line into L2.
+    // `row` is the statistic row of the cursor's (layer, head): it is looked up (an indexed read of the kernel
+    // parameters) only when the stream changes, never on the per-step path.
+    constexpr int kStatAhead = 12;
+    struct Cursor {
+      int it = 0, qi = 0, g = 0, li = 0;
+      const float* row = nullptr;
+    };
+    auto row_of = [&](int li, int g) {
+      const int slot = slot0 + (li < n_layers ? li : 0);
+      const float* src = stat_kind == 0 ? p.lse[slot] : p.delta[slot];
+      return src + (size_t(b) * p.Hq + hk * G + g) * p.S;
+    };
+    auto advance = [&](Cursor& c) {
+      ++c.it;
+      if (++c.qi == per_stream) {
+        c.qi = 0;
+        if (++c.g == G) {
+          c.g = 0;
+          ++c.li;
+        }
+        c.row = row_of(c.li, c.g);
+      }
+    };
+    auto locate = [&](const Cursor& c, bool& valid) {  // address of this thread's statistic of step c (clamped, always valid)
+      const int qc = (qt_first + c.qi) * BQ2 + stat_col;
+      valid = c.it < n_iter && qc < p.S;
+      return c.row + (valid ? qc : p.S - 1);
+    };
+    Cursor cf, cp;
+    cf.row = cp.row = row_of(0, 0);
+    for (int i = 0; i < kStatAhead; ++i) advance(cp);
+    auto request = [&]() -> bool {  // cp.async of the next step's value into its ring slot; returns its validity
+      bool ahead_valid, valid;
+      const float* ahead = locate(cp, ahead_valid);
+      if ((stat_col & 31) == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(ahead));
+      advance(cp);
+      const float* ptr = locate(cf, valid);
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(raw + (cf.it & 7) * 128)), "l"(ptr) : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      advance(cf);
+      return valid;
+    };
+    auto stage = [&](int step, bool valid) {  // the value of `step` has landed: split it into the step's operand tile
+      *reinterpret_cast<uint4*>(stat_row + (step & 3) * 2048) = split3_bf16(valid ? raw[(step & 7) * 128] * stat_mul : stat_pad);
+    };
+    // validity flags of the requests in flight, oldest (step it+3) in bit 0
+    uint32_t vbits = 0;
+    {
+      const bool a0 = request(), a1 = request(), a2 = request();
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      stage(0, a0);
+      stage(1, a1);
+      stage(2, a2);
+      // steps 3..7; from here on a ring slot is requested again only after its previous value has been staged
+#pragma unroll
+      for (int i = 0; i < 5; ++i) vbits |= uint32_t(request()) << i;
+    }
+    fence_proxy_async_smem();
+    mbar_arrive(stat0);
     int li = 0, g = 0, qi = 0;
     bool ok = true;
     for (int it = 0; it < n_iter; ++it) {
@@ -532,6 +524,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 1) bwd_kernel(const __grid_consta
       tmem_ld_x32(tm_dq + lane_sel, a);
       tmem_ld_x32(tm_dq + lane_sel + 32, c);
       tmem_ld_wait();
+      // The operand tile of step it+3 (last read by the scores of step it-1, which completed before this step's
+      // dQ^T did) and the request for step it+8.  The arrival below publishes the tile: the issuing warp waits for
+      // it before the next step's dQ^T, a whole step before the scores of step it+3 are issued.
+      vbits |= uint32_t(request()) << 5;
+      asm volatile("cp.async.wait_group 5;" ::: "memory");
+      stage(it + 3, vbits & 1u);
+      vbits >>= 1;
+      fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(dq_free);
       if (active) {

@@ -38,7 +38,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum): STORED CONSTANTS, not measured by this
 # program.  They come from ncu captures of the small case of each kernel, scaled to a full-size launch by the units
 # one launch processes (traffic grows in proportion); the committed profile summaries give the captures and dates.
-NCU_TRAFFIC_BYTES = {"bwd_kernel": None, "attn_fwd_kernel": 0.474e9, "decode_kernel": 77.96e9}
+NCU_TRAFFIC_BYTES = {"bwd_kernel": 7.45e9, "attn_fwd_kernel": 0.474e9, "decode_kernel": 77.96e9}
 NCU_TRAFFIC_NOTE = "bytes per launch; a stored constant from an earlier ncu capture, not measured in this run"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -500,7 +500,7 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
                 "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS, "kernels": per_kernel}
     # end to end through the public API with host buffers
     e2e_obj, block_e2e = None, None
-    if e2e and not args.small:
+    if e2e and not args.small and not args.no_e2e:
         e2e_steps = max(3, min(args.steps, 5))
         for mode in ("attn", "block"):
             runner.setup_e2e(mode)
@@ -583,7 +583,7 @@ def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, st
     achieved = step_bytes / (k_ms * 1e-3) / 1e9
     peak = peaks["hbm_gbs"]
     unshared_bytes = W.decode_step_bytes(W.C3_UNSHARED, [mean_len] * cfg.B)
-    if args.small:
+    if args.small or args.no_e2e:
         ms_e2e, e2e_steps = float("nan"), 1
         runner.h2d = runner.d2h = 0
     else:
@@ -597,7 +597,7 @@ def run_decode(args, kvp, rank, local_rank, world, device, peaks, peaks_kind, st
     # the two other report modes: the same model decoded layer by layer (consumers re-read their donor's pages), and
     # the same model with nothing shared (every layer stores and reads its own K/V); a bounded number of steps each
     modes = {}
-    if not args.small and extra_modes:
+    if not args.small and extra_modes and not args.no_e2e:
         m_steps = min(steps, 32)
         unshared_m = W.decode_step_bytes(W.C3_UNSHARED, [float(lens0.double().mean()) + (m_steps + 1) / 2.0] * cfg.B)
         for key, mcfg, per_layer in (("per_layer_sequential", cfg, True), ("unshared", W.C3_UNSHARED, False)):
@@ -968,6 +968,8 @@ def main():
     ap.add_argument("--no-decode", action="store_true", help="skip the decode workload in the default run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the shortened prefill and tail-stage runs of the default line")
+    ap.add_argument("--no-e2e", action="store_true",
+                    help="skip the end-to-end arms and the extra decode modes (for profiler launch lists: fewer launches)")
     ap.add_argument("--small", action="store_true",
                     help="reduced shapes of the same kernels (inputs still larger than L2, under 2 GB on the device) "
                          "for profiler captures; implies --no-decode for train and --no-cpu-baseline")

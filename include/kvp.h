@@ -213,8 +213,12 @@ int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal, float sca
 
 /* Chain rule of Eq. 2-3.  dq[l] (bf16) per layer; dk_sum[d], dv_sum[d] (fp32 [B,S,Hkv,dh], owners
  * only) are the sums over the donor, all its consumers and the Hq/Hkv query heads of each KV head,
- * accumulated in fp32 on chip and written once.  At most 8 layers may share one donor.
- * Workspace: kvp_workspace_bytes(KVP_OP_ATTN_BWD). */
+ * accumulated in fp32 on chip across layers, heads and query tiles.  The scores are computed once per
+ * tile pair for all three gradients; partial sums that different thread blocks own (dq over key tiles, dk_sum /
+ * dv_sum over windows of query tiles) are combined by fp32 reductions in global memory, so these outputs are
+ * reproducible up to fp32 summation order, not bit for bit.  dk_sum / dv_sum are overwritten (cleared first),
+ * never accumulated into.  At most 8 layers may share one donor.
+ * Workspace: kvp_workspace_bytes(KVP_OP_ATTN_BWD): Delta per layer plus fp32 dq accumulators for up to 8 layers. */
 int kvp_attn_bwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
                  const void* const* k, const void* const* v, const void* const* o, const void* const* d_o,
                  const float* const* lse, void* const* dq, float* const* dk_sum, float* const* dv_sum, void* ws,

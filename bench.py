@@ -454,8 +454,8 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
     n_groups, n_own = len(cfg.owners()), len(cfg.owners())
     pairs = cfg.S * (cfg.S + 1) // 2
     unit = 2 * cfg.dh * pairs * cfg.B * cfg.Hq * cfg.L        # one attention GEMM over every layer
-    n_gemm = (cfg.L + 2 * n_own) + ((2 * cfg.L + 2 * n_own) if backward else 0)
-    # kernel -> (timed event pairs per step, algorithmic FLOPs per step, executed FLOPs per step)
+    n_gemm = (cfg.L + 2 * n_own) + ((2 * cfg.L + 2 * n_own) if backward else 0)   # GEMM problems; launches are fewer
+    # kernel -> (event pairs to provide per step, algorithmic FLOPs per step, executed FLOPs per step)
     kernels = {"attn_fwd_kernel": (kvp.KERNEL_ATTN_FWD, cfg.L, 2 * unit, 2 * unit),
                "gemm_kernel": (kvp.KERNEL_GEMM, n_gemm, runner.gemm_flops(), runner.gemm_flops())}
     if backward:
@@ -476,9 +476,11 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
     block_tflops = world * flops / (ms_step * 1e-3) / 1e12
     peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
     per_kernel = {}
-    for name, (kid, n, algo, execd) in kernels.items():
-        k_ms = sum(timers[name].durations_ms()) / args.steps
-        per_kernel[name] = {"timed_launch_groups_per_step": n, "ms_per_step": k_ms, "share_of_step": k_ms / ms_step,
+    for name, (kid, _n, algo, execd) in kernels.items():
+        durs = timers[name].durations_ms()
+        k_ms = sum(durs) / args.steps
+        per_kernel[name] = {"timed_launch_groups_per_step": len(durs) / args.steps, "ms_per_step": k_ms,
+                            "share_of_step": k_ms / ms_step,
                             "algorithmic_tflops": algo / (k_ms * 1e-3) / 1e12,
                             "executed_tflops": execd / (k_ms * 1e-3) / 1e12}
     attn_names = [n for n in per_kernel if n != "gemm_kernel"]
@@ -493,7 +495,7 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
                 "frac": achieved / peak, "traffic": traffic,
                 "traffic_unit": NCU_TRAFFIC_NOTE,
                 "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
-                "launches_per_step": n_groups if top == "bwd_kernel" else per_kernel[top]["timed_launch_groups_per_step"],
+                "launches_per_step": per_kernel[top]["timed_launch_groups_per_step"],
                 "kernel_ms_per_step": per_kernel[top]["ms_per_step"],
                 "share_of_step": per_kernel[top]["share_of_step"],
                 "executed_tflops": per_kernel[top]["executed_tflops"],
@@ -880,15 +882,27 @@ def run_stage_fwd(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)
     D, H, dh, S = 4096, 32, 128, 8192
     full = W.TrainCfg("stage-mha-unconverted", 4, 1, S, D, H, H, dh, [0, 1, 2, 3])
     local = W.TrainCfg("stage-mha-local-donor", 4, 1, S, D, H, H, dh, [0, 0, 0, 0])
-    res = {}
-    for name, cfg, lm in (("regular", full, False), ("tail", full, True), ("tail_converted", local, True)):
-        r = StageFwdRunner(kvp, cfg, device, lm_head=lm)
-        for i in range(max(args.warmup, 40)):       # long enough for the power-capped clock to settle
+    # The three stage kinds are timed in turn, round after round, and each reports the median of its rounds: the
+    # SM clock under the power cap drifts over seconds, and back-to-back blocks would put that drift into the ratios.
+    kinds = (("regular", full, False), ("tail", full, True), ("tail_converted", local, True))
+    runners = {name: StageFwdRunner(kvp, cfg, device, lm_head=lm) for name, cfg, lm in kinds}
+    for i in range(max(args.warmup, 20)):           # long enough for the power-capped clock to settle
+        for r in runners.values():
             r.step(i)
-        ms, clocks = timed_region(r.step, args.steps, device, local_rank)
-        res[name] = {"ms": ms / args.steps, "elementwise_bytes": r.elem_bytes, "sm_mhz": clocks.get("sm_mhz")}
-        del r
-        torch.cuda.empty_cache()
+    rounds, per_round = 7, max(args.steps, 4)
+    samples = {name: [] for name in runners}
+    mhz = {name: [] for name in runners}
+    for _ in range(rounds):
+        for name, r in runners.items():
+            ms, clocks = timed_region(r.step, per_round, device, local_rank)
+            samples[name].append(ms / per_round)
+            if clocks.get("sm_mhz") is not None:
+                mhz[name].append(clocks["sm_mhz"])
+    res = {name: {"ms": float(np.median(samples[name])), "ms_min": min(samples[name]), "ms_max": max(samples[name]),
+                  "rounds": rounds, "steps_per_round": per_round, "elementwise_bytes": runners[name].elem_bytes,
+                  "sm_mhz": float(np.median(mhz[name])) if mhz[name] else None} for name in runners}
+    del runners
+    torch.cuda.empty_cache()
     # the element-wise kernels alone, against the measured copy bandwidth
     r = StageFwdRunner(kvp, full, device)
     T, F = full.T, r.F

@@ -175,7 +175,8 @@ size_t kvp_workspace_bytes(int op, const kvp_shape* s, const int32_t* donor);
 
 /* Eq. 1.  q[l] = x[l] wq[l]^T for every layer; k[l] = x[l] wk[l]^T, v[l] = x[l] wv[l]^T for owners
  * only (Eq. 3 removes them for consumers).  x[l]: [B*S, D]; wq[l]: [Hq*dh, D]; wk[l], wv[l]:
- * [Hkv*dh, D]; q[l]: [B,S,Hq,dh]; k[l], v[l]: [B,S,Hkv,dh]. */
+ * [Hkv*dh, D]; q[l]: [B,S,Hq,dh]; k[l], v[l]: [B,S,Hkv,dh].  All projections of all layers are tiles of one
+ * grouped GEMM launch (one launch per 32 projections). */
 int kvp_proj_fwd(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
                  const void* const* wk, const void* const* wv, void* const* q, void* const* k, void* const* v,
                  void* ws, size_t ws_bytes, kvp_stream_t stream);
@@ -183,7 +184,9 @@ int kvp_proj_fwd(const kvp_shape* s, const int32_t* donor, const void* const* x,
 /* Chain rule of Eq. 1.  dwq[l] = dq[l]^T x[l] (fp32 [Hq*dh, D]); dx[l] = dq[l] wq[l] (bf16 [B*S, D]);
  * owners add dwk = dk_sum^T x, dwv = dv_sum^T x and dx += dk_sum wk + dv_sum wv, where dk_sum, dv_sum
  * (fp32 [B,S,Hkv,dh]) are the donor-group sums written by kvp_attn_bwd, rounded once to bf16.
- * Workspace: kvp_workspace_bytes(KVP_OP_PROJ_BWD, ...). */
+ * Layers are taken eight at a time: the sums of the eight layers' owners are rounded into the workspace, then one
+ * grouped GEMM launch writes every gradient of those layers.
+ * Workspace: kvp_workspace_bytes(KVP_OP_PROJ_BWD, ...) = bf16 copies of dk_sum and dv_sum for min(owners, 8) layers. */
 int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
                  const void* const* wk, const void* const* wv, const void* const* dq, const float* const* dk_sum,
                  const float* const* dv_sum, float* const* dwq, float* const* dwk, float* const* dwv,

@@ -1,5 +1,6 @@
 // C-ABI entry points of the training / prefill path: argument validation and the sequence of
 // kernel launches per layer.  No allocation, no synchronisation.
+#include <algorithm>
 #include <vector>
 
 #include "kvp_host.h"
@@ -121,12 +122,32 @@ Sizes sizes_of(const kvp_shape* s) {
   return Sizes{{T * D, false}, {nq * D, false}, {nkv * D, true}, {T * nq, false}, {T * nkv, true}};
 }
 
+// Layers per grouped launch of the projection backward: 8 layers are at most 32 problems and 48 operand pairs.
+constexpr int kProjBwdChunk = 8;
+
+GemmProblem problem(int M, int N, GemmSeg seg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32) {
+  GemmProblem g{};
+  g.M = M;
+  g.N = N;
+  g.segs[0] = seg;
+  g.nseg = 1;
+  g.a_mn = a_mn;
+  g.b_mn = b_mn;
+  g.c = c;
+  g.ldc = ldc;
+  g.out_f32 = out_f32;
+  return g;
+}
+
 // scratch the bf16 form of an operation needs (before any shadows)
 size_t op_scratch_bytes(int op, const kvp_shape* s, const int32_t* donor) {
   switch (op) {
-    case KVP_OP_PROJ_BWD:
-      // bf16 copies of one owner's dk_sum and dv_sum
-      return 2 * align256(size_t(s->B) * s->S * s->Hkv * s->dh * 2);
+    case KVP_OP_PROJ_BWD: {
+      // bf16 copies of dk_sum and dv_sum of the owners of one chunk of layers
+      int owners = 0;
+      for (int l = 0; l < s->L; ++l) owners += donor[l] == l;
+      return size_t(2 * std::min(owners, kProjBwdChunk)) * align256(size_t(s->B) * s->S * s->Hkv * s->dh * 2);
+    }
     case KVP_OP_ATTN_BWD:
       return attn_bwd_workspace(s, donor);
     default:
@@ -198,20 +219,16 @@ extern "C" int kvp_proj_fwd(const kvp_shape* s, const int32_t* donor, const void
     return rc != KVP_OK ? rc : sh.finish();
   }
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh, Nkv = s->Hkv * s->dh;
+  // Every projection of every layer in one grouped launch; consumers have no K/V projections (Eq. 3).
+  std::vector<GemmProblem> probs;
+  probs.reserve(size_t(3) * s->L);
+  for (int l = 0; l < s->L; ++l) probs.push_back(problem(T, Nq, {x[l], wq[l], D, D, D}, 0, 0, q[l], Nq, 0));
   for (int l = 0; l < s->L; ++l) {
-    GemmSeg sq{x[l], wq[l], D, D, D};
-    rc = gemm_bf16(T, Nq, &sq, 1, 0, 0, q[l], Nq, 0, stream);
-    if (rc != KVP_OK) return rc;
-    if (donor[l] == l) {  // consumers have no K/V projections (Eq. 3)
-      GemmSeg sk{x[l], wk[l], D, D, D};
-      rc = gemm_bf16(T, Nkv, &sk, 1, 0, 0, k[l], Nkv, 0, stream);
-      if (rc != KVP_OK) return rc;
-      GemmSeg sv{x[l], wv[l], D, D, D};
-      rc = gemm_bf16(T, Nkv, &sv, 1, 0, 0, v[l], Nkv, 0, stream);
-      if (rc != KVP_OK) return rc;
-    }
+    if (donor[l] != l) continue;
+    probs.push_back(problem(T, Nkv, {x[l], wk[l], D, D, D}, 0, 0, k[l], Nkv, 0));
+    probs.push_back(problem(T, Nkv, {x[l], wv[l], D, D, D}, 0, 0, v[l], Nkv, 0));
   }
-  return KVP_OK;
+  return gemm_grouped(probs.data(), int(probs.size()), stream);
 }
 
 extern "C" int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
@@ -261,30 +278,45 @@ extern "C" int kvp_proj_bwd_range(const kvp_shape* s, const int32_t* donor, cons
   }
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh, Nkv = s->Hkv * s->dh;
   const size_t n_kv = size_t(T) * Nkv;
-  uint8_t* dk_bf = reinterpret_cast<uint8_t*>(ws);
-  uint8_t* dv_bf = dk_bf + align256(n_kv * 2);
-  for (int l = layer_begin; l < layer_end; ++l) {
-    // dWq = dQ^T X : A = dQ stored [T, Nq] (MN-major for M = Nq), B = X stored [T, D] (MN-major for N = D)
-    GemmSeg swq{dq[l], x[l], Nq, D, T};
-    rc = gemm_bf16(Nq, D, &swq, 1, 1, 1, dwq[l], D, 1, stream);
-    if (rc != KVP_OK) return rc;
-    if (donor[l] == l) {
-      rc = cast_f32_to_bf16(dk_sum[l], dk_bf, n_kv, stream);
-      if (rc == KVP_OK) rc = cast_f32_to_bf16(dv_sum[l], dv_bf, n_kv, stream);
+  const size_t slot = align256(n_kv * 2);
+  uint8_t* bf = reinterpret_cast<uint8_t*>(ws);
+  // Chunks of up to kProjBwdChunk layers: the fp32 donor-group sums of the chunk's owners are rounded to bf16 into
+  // the workspace, then ONE grouped launch produces every gradient of the chunk.  The weight gradients come first
+  // in the list (their tiles run over all T tokens, the longest), then dX = dQ Wq + dK Wk + dV Wv of the owners
+  // (three K segments into one accumulator), then the consumers' dX = dQ Wq.
+  std::vector<GemmProblem> probs;
+  for (int c0 = layer_begin; c0 < layer_end; c0 += kProjBwdChunk) {
+    const int c1 = std::min(layer_end, c0 + kProjBwdChunk);
+    probs.clear();
+    std::vector<uint8_t*> dk_bf(size_t(c1 - c0), nullptr), dv_bf(size_t(c1 - c0), nullptr);
+    int owners = 0;
+    for (int l = c0; l < c1; ++l) {
+      if (donor[l] != l) continue;
+      dk_bf[l - c0] = bf + size_t(2 * owners) * slot;
+      dv_bf[l - c0] = bf + size_t(2 * owners + 1) * slot;
+      ++owners;
+      rc = cast_f32_to_bf16(dk_sum[l], dk_bf[l - c0], n_kv, stream);
+      if (rc == KVP_OK) rc = cast_f32_to_bf16(dv_sum[l], dv_bf[l - c0], n_kv, stream);
       if (rc != KVP_OK) return rc;
-      GemmSeg swk{dk_bf, x[l], Nkv, D, T};
-      rc = gemm_bf16(Nkv, D, &swk, 1, 1, 1, dwk[l], D, 1, stream);
-      if (rc != KVP_OK) return rc;
-      GemmSeg swv{dv_bf, x[l], Nkv, D, T};
-      rc = gemm_bf16(Nkv, D, &swv, 1, 1, 1, dwv[l], D, 1, stream);
-      if (rc != KVP_OK) return rc;
-      // dX = dQ Wq + dK Wk + dV Wv in one pass: three K segments into the same accumulator
-      GemmSeg segs[3] = {{dq[l], wq[l], Nq, D, Nq}, {dk_bf, wk[l], Nkv, D, Nkv}, {dv_bf, wv[l], Nkv, D, Nkv}};
-      rc = gemm_bf16(T, D, segs, 3, 0, 1, dx[l], D, 0, stream);
-    } else {
-      GemmSeg sx{dq[l], wq[l], Nq, D, Nq};
-      rc = gemm_bf16(T, D, &sx, 1, 0, 1, dx[l], D, 0, stream);
     }
+    // dWq = dQ^T X : A = dQ stored [T, Nq] (MN-major for M = Nq), B = X stored [T, D] (MN-major for N = D)
+    for (int l = c0; l < c1; ++l) probs.push_back(problem(Nq, D, {dq[l], x[l], Nq, D, T}, 1, 1, dwq[l], D, 1));
+    for (int l = c0; l < c1; ++l) {
+      if (donor[l] != l) continue;
+      probs.push_back(problem(Nkv, D, {dk_bf[l - c0], x[l], Nkv, D, T}, 1, 1, dwk[l], D, 1));
+      probs.push_back(problem(Nkv, D, {dv_bf[l - c0], x[l], Nkv, D, T}, 1, 1, dwv[l], D, 1));
+    }
+    for (int l = c0; l < c1; ++l) {
+      if (donor[l] != l) continue;
+      GemmProblem g = problem(T, D, {dq[l], wq[l], Nq, D, Nq}, 0, 1, dx[l], D, 0);
+      g.segs[1] = {dk_bf[l - c0], wk[l], Nkv, D, Nkv};
+      g.segs[2] = {dv_bf[l - c0], wv[l], Nkv, D, Nkv};
+      g.nseg = 3;
+      probs.push_back(g);
+    }
+    for (int l = c0; l < c1; ++l)
+      if (donor[l] != l) probs.push_back(problem(T, D, {dq[l], wq[l], Nq, D, Nq}, 0, 1, dx[l], D, 0));
+    rc = gemm_grouped(probs.data(), int(probs.size()), stream);
     if (rc != KVP_OK) return rc;
   }
   return KVP_OK;
@@ -298,13 +330,12 @@ extern "C" int kvp_out_proj_fwd(const kvp_shape* s, const void* const* o, const 
   if (o == nullptr || wo == nullptr || y == nullptr) return KVP_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh;
+  std::vector<GemmProblem> probs;
   for (int l = 0; l < s->L; ++l) {
     if (o[l] == nullptr || wo[l] == nullptr || y[l] == nullptr) return KVP_ERR_INVALID_ARG;
-    GemmSeg sg{o[l], wo[l], Nq, Nq, Nq};
-    rc = gemm_bf16(T, D, &sg, 1, 0, 0, y[l], D, 0, stream);
-    if (rc != KVP_OK) return rc;
+    probs.push_back(problem(T, D, {o[l], wo[l], Nq, Nq, Nq}, 0, 0, y[l], D, 0));
   }
-  return KVP_OK;
+  return gemm_grouped(probs.data(), int(probs.size()), stream);
 }
 
 extern "C" int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const void* const* wo,
@@ -315,19 +346,15 @@ extern "C" int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const 
   if (o == nullptr || wo == nullptr || dy == nullptr || d_o == nullptr || dwo == nullptr) return KVP_ERR_INVALID_ARG;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   const int T = s->B * s->S, D = s->D, Nq = s->Hq * s->dh;
-  for (int l = 0; l < s->L; ++l) {
+  std::vector<GemmProblem> probs;
+  for (int l = 0; l < s->L; ++l)
     if (o[l] == nullptr || wo[l] == nullptr || dy[l] == nullptr || d_o[l] == nullptr || dwo[l] == nullptr)
       return KVP_ERR_INVALID_ARG;
-    // dO = dY Wo : A = dY [T, D] K-major, B = Wo stored [D, Nq] = [K, N] (MN-major)
-    GemmSeg s1{dy[l], wo[l], D, Nq, D};
-    rc = gemm_bf16(T, Nq, &s1, 1, 0, 1, d_o[l], Nq, 0, stream);
-    if (rc != KVP_OK) return rc;
-    // dWo = dY^T O : [D, Nq], both operands stored token-major
-    GemmSeg s2{dy[l], o[l], D, Nq, T};
-    rc = gemm_bf16(D, Nq, &s2, 1, 1, 1, dwo[l], Nq, 1, stream);
-    if (rc != KVP_OK) return rc;
-  }
-  return KVP_OK;
+  // dWo = dY^T O : [D, Nq], both operands stored token-major (the longest tiles: first in the list)
+  for (int l = 0; l < s->L; ++l) probs.push_back(problem(D, Nq, {dy[l], o[l], D, Nq, T}, 1, 1, dwo[l], Nq, 1));
+  // dO = dY Wo : A = dY [T, D] K-major, B = Wo stored [D, Nq] = [K, N] (MN-major)
+  for (int l = 0; l < s->L; ++l) probs.push_back(problem(T, Nq, {dy[l], wo[l], D, Nq, D}, 0, 1, d_o[l], Nq, 0));
+  return gemm_grouped(probs.data(), int(probs.size()), stream);
 }
 
 extern "C" int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,

@@ -8,6 +8,9 @@
 // MN-major in memory; that only changes the TMA box and the shared-memory descriptor.
 // The K extent may be split over up to three operand pairs ("segments") that accumulate into the
 // same tile, which is how dX = dQ Wq + dK Wk + dV Wv is produced with one output pass.
+// One launch walks the tiles of a whole list of problems (different shapes, operands, operand modes and output
+// types): the Q, K and V projections of every layer are one launch, so are all weight and input gradients of a
+// backward pass, and the SMs idle only behind the last tile of the list instead of behind each GEMM's last wave.
 #include "kvp_host.h"
 #include "kvp_sm100.cuh"
 
@@ -22,25 +25,48 @@ constexpr int GEMM_THREADS = 192;
 constexpr int MAX_SEG = 3;
 constexpr int GROUP_M = 16;  // m-tiles per rasterisation group (keeps an A slab resident in L2)
 constexpr size_t GEMM_SMEM = 1024 + size_t(STAGES) * STAGE_BYTES + 256;
+constexpr int MAX_PROB = 32;   // problems per launch
+constexpr int MAX_MAPS = 96;   // tensor maps per launch (two per segment)
 
 __device__ int g_gemm_status;
 
-struct GemmParams {
-  CUtensorMap map_a[MAX_SEG];
-  CUtensorMap map_b[MAX_SEG];
-  int kblocks[MAX_SEG];  // k-blocks (of BK) per segment
-  int nseg;
+struct Problem {
   int M, N;
+  int m_tiles, n_tiles;
+  int tile_end;            // one past this problem's last tile in the launch's tile order
+  int nseg;
+  int kblocks[MAX_SEG];    // k-blocks (of BK) per segment
+  int total_kb;
+  short map_a[MAX_SEG];    // indices into GemmParams::maps
+  short map_b[MAX_SEG];
   int a_mn, b_mn;
   int out_f32;
+  uint32_t idesc;
   long long ldc;
   void* c;
-  uint32_t idesc;
+};
+
+struct GemmParams {
+  CUtensorMap maps[MAX_MAPS];
+  Problem prob[MAX_PROB];
+  int nprob;
+  int total_tiles;
   // Self-test of the bounded waits (0 in every ordinary launch): the k-block count, plus one, at which the MMA
   // warp of CTA 0 withholds the arrival that frees a ring stage, and the wait limit that launch runs with.
   int withhold_at;
   unsigned long long wait_limit_ns;
 };
+
+// Position of tile t inside its problem: groups of GROUP_M m-tiles are walked n-tile by n-tile, which keeps an
+// A slab resident in L2 while the B tiles stream past it.
+__device__ __forceinline__ void tile_coords(int within_problem, int m_tiles, int n_tiles, int& tm, int& tn) {
+  const int per_group = GROUP_M * n_tiles;
+  const int g = within_problem / per_group;
+  const int within = within_problem - g * per_group;
+  const int gm = min(GROUP_M, m_tiles - g * GROUP_M);
+  tm = g * GROUP_M + within % gm;
+  tn = within / gm;
+}
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -55,12 +81,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   int* err = &g_gemm_status;
-
-  const int m_tiles = (p.M + BM - 1) / BM;
-  const int n_tiles = (p.N + BN - 1) / BN;
-  const int total_tiles = m_tiles * n_tiles;
-  int total_kb = 0;
-  for (int s = 0; s < p.nseg; ++s) total_kb += p.kblocks[s];
+  const int total_tiles = p.total_tiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -82,33 +103,25 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  auto tile_coords = [&](int t, int& tm, int& tn) {
-    const int per_group = GROUP_M * n_tiles;
-    const int g = t / per_group;
-    const int within = t - g * per_group;
-    const int gm = min(GROUP_M, m_tiles - g * GROUP_M);
-    tm = g * GROUP_M + within % gm;
-    tn = within / gm;
-  };
-
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     {
       const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
-      if (lane == 0)
-        for (int s = 0; s < p.nseg; ++s) {
-          tma_prefetch_desc(&p.map_a[s]);
-          tma_prefetch_desc(&p.map_b[s]);
-        }
-      __syncwarp();
       uint32_t it = 0;
       bool ok = true;
+      int pi = 0;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        while (t >= p.prob[pi].tile_end) ++pi;
+        const Problem& pr = p.prob[pi];
         int tm, tn;
-        tile_coords(t, tm, tn);
+        tile_coords(t - (pi ? p.prob[pi - 1].tile_end : 0), pr.m_tiles, pr.n_tiles, tm, tn);
         const int m0 = tm * BM, n0 = tn * BN;
-        for (int seg = 0; seg < p.nseg && ok; ++seg) {
-          for (int kb = 0; kb < p.kblocks[seg]; ++kb, ++it) {
+        const int a_mn = pr.a_mn, b_mn = pr.b_mn;
+        for (int seg = 0; seg < pr.nseg && ok; ++seg) {
+          const CUtensorMap* map_a = &p.maps[pr.map_a[seg]];
+          const CUtensorMap* map_b = &p.maps[pr.map_b[seg]];
+          const int nkb = pr.kblocks[seg];
+          for (int kb = 0; kb < nkb; ++kb, ++it) {
             const int s = it % STAGES;
             const uint32_t ph = (it / STAGES) & 1;
             if (!mbar_wait(&empty[s], ph ^ 1, err, p.wait_limit_ns)) { ok = false; break; }
@@ -116,17 +129,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
             uint8_t* sb = sa + A_BYTES;
             mbar_expect_tx_e(&full[s], STAGE_BYTES, leader);
             const int k0 = kb * BK;
-            if (p.a_mn == 0) {
-              tma_load_2d_e(sa, &p.map_a[seg], &full[s], k0, m0, leader);
+            if (a_mn == 0) {
+              tma_load_2d_e(sa, map_a, &full[s], k0, m0, leader);
             } else {
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j) tma_load_2d_e(sa + j * 8192, &p.map_a[seg], &full[s], m0 + 64 * j, k0, leader);
+              for (int j = 0; j < BM / 64; ++j) tma_load_2d_e(sa + j * 8192, map_a, &full[s], m0 + 64 * j, k0, leader);
             }
-            if (p.b_mn == 0) {
-              tma_load_2d_e(sb, &p.map_b[seg], &full[s], k0, n0, leader);
+            if (b_mn == 0) {
+              tma_load_2d_e(sb, map_b, &full[s], k0, n0, leader);
             } else {
 #pragma unroll
-              for (int j = 0; j < BN / 64; ++j) tma_load_2d_e(sb + j * 8192, &p.map_b[seg], &full[s], n0 + 64 * j, k0, leader);
+              for (int j = 0; j < BN / 64; ++j) tma_load_2d_e(sb + j * 8192, map_b, &full[s], n0 + 64 * j, k0, leader);
             }
           }
         }
@@ -139,11 +152,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       uint32_t it = 0;
       uint32_t tile_i = 0;
       bool ok = true;
-      const uint32_t a_step = p.a_mn ? 2048u : 32u;   // bytes per 16-deep K step
-      const uint32_t b_step = p.b_mn ? 2048u : 32u;
-      const uint32_t a_lbo = p.a_mn ? 8192u : 0u;
-      const uint32_t b_lbo = p.b_mn ? 8192u : 0u;
+      int pi = 0;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
+        while (t >= p.prob[pi].tile_end) ++pi;
+        const Problem& pr = p.prob[pi];
+        const uint32_t a_step = pr.a_mn ? 2048u : 32u;   // bytes per 16-deep K step
+        const uint32_t b_step = pr.b_mn ? 2048u : 32u;
+        const uint32_t a_lbo = pr.a_mn ? 8192u : 0u;
+        const uint32_t b_lbo = pr.b_mn ? 8192u : 0u;
+        const uint32_t idesc = pr.idesc;
+        const int total_kb = pr.total_kb;
         const int acc = tile_i & 1;
         const uint32_t acc_ph = (tile_i >> 1) & 1;
         if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1, err, p.wait_limit_ns)) { ok = false; break; }
@@ -160,7 +178,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = smem_desc_sw128(sa + k * a_step, a_lbo, 1024);
             const uint64_t db = smem_desc_sw128(sb + k * b_step, b_lbo, 1024);
-            umma_ss(d_tmem, da, db, p.idesc, (kb | k) != 0, leader);
+            umma_ss(d_tmem, da, db, idesc, (kb | k) != 0, leader);
           }
           // frees the smem stage once these MMAs have read it
           if (!(p.withhold_at != 0 && blockIdx.x == 0 && it + 1 == uint32_t(p.withhold_at))) umma_commit(&empty[s], leader);
@@ -172,9 +190,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     // ------------------------------ epilogue (warps 2..5) ------------------------------
     const int quarter = warp & 3;  // TMEM lane quarter this warp may access
     uint32_t tile_i = 0;
+    int pi = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++tile_i) {
+      while (t >= p.prob[pi].tile_end) ++pi;
+      const Problem& pr = p.prob[pi];
       int tm, tn;
-      tile_coords(t, tm, tn);
+      tile_coords(t - (pi ? p.prob[pi - 1].tile_end : 0), pr.m_tiles, pr.n_tiles, tm, tn);
+      const int M = pr.M, N = pr.N, out_f32 = pr.out_f32;
+      const long long ldc = pr.ldc;
+      void* const c = pr.c;
       const int acc = tile_i & 1;
       const uint32_t acc_ph = (tile_i >> 1) & 1;
       bool ok = mbar_wait(&acc_full[acc], acc_ph, err, p.wait_limit_ns);
@@ -185,25 +209,25 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * BN;
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (n0 + c0 >= p.N) break;  // uniform across the warp
+        if (n0 + c0 >= N) break;  // uniform across the warp
         uint32_t r[32];
         tmem_ld_x32(taddr + c0, r);
         tmem_ld_wait();
-        if (row < p.M) {
-          if (p.out_f32) {
-            float* dst = reinterpret_cast<float*>(p.c) + size_t(row) * p.ldc + n0 + c0;
+        if (row < M) {
+          if (out_f32) {
+            float* dst = reinterpret_cast<float*>(c) + size_t(row) * ldc + n0 + c0;
 #pragma unroll
             for (int v = 0; v < 8; ++v) {
-              if (n0 + c0 + v * 4 < p.N) {
+              if (n0 + c0 + v * 4 < N) {
                 uint4 val = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
                 *reinterpret_cast<uint4*>(dst + v * 4) = val;
               }
             }
           } else {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.c) + size_t(row) * p.ldc + n0 + c0;
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(c) + size_t(row) * ldc + n0 + c0;
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
-              if (n0 + c0 + v * 8 < p.N) {
+              if (n0 + c0 + v * 8 < N) {
                 uint4 val;
                 val.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
                 val.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
@@ -242,69 +266,135 @@ int gemm_read_status() {
   return v;
 }
 
-int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32,
-              cudaStream_t stream, int withhold_at, unsigned long long wait_limit_ns) {
-  if (M <= 0 || N <= 0 || nseg < 1 || nseg > MAX_SEG || c == nullptr) return KVP_ERR_INVALID_ARG;
-  if ((N % 8) != 0 || (ldc % 8) != 0 || !aligned16(c)) return KVP_ERR_UNSUPPORTED;
-  GemmParams p;
-  p.nseg = nseg;
-  p.M = M;
-  p.N = N;
-  p.a_mn = a_mn;
-  p.b_mn = b_mn;
-  p.out_f32 = out_f32;
-  p.ldc = ldc;
-  p.c = c;
-  p.idesc = umma_idesc_bf16(BM, BN, a_mn, b_mn);
+namespace {
+
+int check_problem(const GemmProblem& g) {
+  if (g.M <= 0 || g.N <= 0 || g.nseg < 1 || g.nseg > MAX_SEG || g.c == nullptr) return KVP_ERR_INVALID_ARG;
+  if ((g.N % 8) != 0 || (g.ldc % 8) != 0 || !aligned16(g.c)) return KVP_ERR_UNSUPPORTED;
+  for (int s = 0; s < g.nseg; ++s) {
+    const GemmSeg& e = g.segs[s];
+    if (e.a == nullptr || e.b == nullptr || e.K <= 0) return KVP_ERR_INVALID_ARG;
+    if ((e.K % 8) != 0 || (e.lda % 8) != 0 || (e.ldb % 8) != 0 || !aligned16(e.a) || !aligned16(e.b))
+      return KVP_ERR_UNSUPPORTED;
+  }
+  return KVP_OK;
+}
+
+// Tensor maps of one operand pair; the box depends on the operand mode only.
+int encode_segment(const GemmProblem& g, const GemmSeg& e, CUtensorMap* map_a, CUtensorMap* map_b) {
+  int rc;
+  if (g.a_mn == 0) {
+    uint64_t dims[2] = {uint64_t(e.K), uint64_t(g.M)};
+    uint64_t strides[1] = {uint64_t(e.lda) * 2};
+    uint32_t box[2] = {BK, BM};
+    rc = make_tensor_map(map_a, e.a, 2, 2, dims, strides, box, true);
+  } else {
+    uint64_t dims[2] = {uint64_t(g.M), uint64_t(e.K)};
+    uint64_t strides[1] = {uint64_t(e.lda) * 2};
+    uint32_t box[2] = {64, BK};
+    rc = make_tensor_map(map_a, e.a, 2, 2, dims, strides, box, true);
+  }
+  if (rc != KVP_OK) return rc;
+  if (g.b_mn == 0) {
+    uint64_t dims[2] = {uint64_t(e.K), uint64_t(g.N)};
+    uint64_t strides[1] = {uint64_t(e.ldb) * 2};
+    uint32_t box[2] = {BK, BN};
+    rc = make_tensor_map(map_b, e.b, 2, 2, dims, strides, box, true);
+  } else {
+    uint64_t dims[2] = {uint64_t(g.N), uint64_t(e.K)};
+    uint64_t strides[1] = {uint64_t(e.ldb) * 2};
+    uint32_t box[2] = {64, BK};
+    rc = make_tensor_map(map_b, e.b, 2, 2, dims, strides, box, true);
+  }
+  return rc;
+}
+
+int launch_group(const GemmProblem* probs, int n, cudaStream_t stream, int withhold_at, unsigned long long wait_limit_ns) {
+  static thread_local GemmParams p;   // 15 KB: kept off the stack
+  p.nprob = n;
   p.withhold_at = withhold_at;
   p.wait_limit_ns = wait_limit_ns != 0 ? wait_limit_ns : kWaitLimitNs;
-  for (int s = 0; s < nseg; ++s) {
-    const GemmSeg& g = segs[s];
-    if (g.a == nullptr || g.b == nullptr || g.K <= 0) return KVP_ERR_INVALID_ARG;
-    if ((g.K % 8) != 0 || (g.lda % 8) != 0 || (g.ldb % 8) != 0 || !aligned16(g.a) || !aligned16(g.b))
-      return KVP_ERR_UNSUPPORTED;
-    p.kblocks[s] = (g.K + BK - 1) / BK;
-    int rc;
-    if (a_mn == 0) {
-      uint64_t dims[2] = {uint64_t(g.K), uint64_t(M)};
-      uint64_t strides[1] = {uint64_t(g.lda) * 2};
-      uint32_t box[2] = {BK, BM};
-      rc = make_tensor_map(&p.map_a[s], g.a, 2, 2, dims, strides, box, true);
-    } else {
-      uint64_t dims[2] = {uint64_t(M), uint64_t(g.K)};
-      uint64_t strides[1] = {uint64_t(g.lda) * 2};
-      uint32_t box[2] = {64, BK};
-      rc = make_tensor_map(&p.map_a[s], g.a, 2, 2, dims, strides, box, true);
+  int n_maps = 0, tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const GemmProblem& g = probs[i];
+    Problem& q = p.prob[i];
+    q.M = g.M;
+    q.N = g.N;
+    q.m_tiles = (g.M + BM - 1) / BM;
+    q.n_tiles = (g.N + BN - 1) / BN;
+    tiles += q.m_tiles * q.n_tiles;
+    q.tile_end = tiles;
+    q.nseg = g.nseg;
+    q.total_kb = 0;
+    for (int s = 0; s < MAX_SEG; ++s) {
+      q.kblocks[s] = 0;
+      q.map_a[s] = q.map_b[s] = 0;
     }
-    if (rc != KVP_OK) return rc;
-    if (b_mn == 0) {
-      uint64_t dims[2] = {uint64_t(g.K), uint64_t(N)};
-      uint64_t strides[1] = {uint64_t(g.ldb) * 2};
-      uint32_t box[2] = {BK, BN};
-      rc = make_tensor_map(&p.map_b[s], g.b, 2, 2, dims, strides, box, true);
-    } else {
-      uint64_t dims[2] = {uint64_t(N), uint64_t(g.K)};
-      uint64_t strides[1] = {uint64_t(g.ldb) * 2};
-      uint32_t box[2] = {64, BK};
-      rc = make_tensor_map(&p.map_b[s], g.b, 2, 2, dims, strides, box, true);
+    for (int s = 0; s < g.nseg; ++s) {
+      q.kblocks[s] = (g.segs[s].K + BK - 1) / BK;
+      q.total_kb += q.kblocks[s];
+      q.map_a[s] = short(n_maps);
+      q.map_b[s] = short(n_maps + 1);
+      const int rc = encode_segment(g, g.segs[s], &p.maps[n_maps], &p.maps[n_maps + 1]);
+      if (rc != KVP_OK) return rc;
+      n_maps += 2;
     }
-    if (rc != KVP_OK) return rc;
+    q.a_mn = g.a_mn;
+    q.b_mn = g.b_mn;
+    q.out_f32 = g.out_f32;
+    q.idesc = umma_idesc_bf16(BM, BN, g.a_mn, g.b_mn);
+    q.ldc = g.ldc;
+    q.c = g.c;
   }
-  for (int s = nseg; s < MAX_SEG; ++s) {
-    p.kblocks[s] = 0;
-    p.map_a[s] = p.map_a[0];
-    p.map_b[s] = p.map_b[0];
-  }
+  for (int i = n; i < MAX_PROB; ++i) p.prob[i] = p.prob[n - 1];
+  p.total_tiles = tiles;
   static const cudaError_t attr =
       cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GEMM_SMEM));
   if (attr != cudaSuccess) return KVP_ERR_CUDA;
-  const int m_tiles = (M + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
-  const int grid = min(m_tiles * n_tiles, sm_count());
+  const int grid = min(tiles, sm_count());
   timing_before(KVP_KERNEL_GEMM, stream);
   gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);
   timing_after(KVP_KERNEL_GEMM, stream);
   note_launch();
   return cudaGetLastError() == cudaSuccess ? KVP_OK : KVP_ERR_CUDA;
+}
+
+}  // namespace
+
+int gemm_grouped(const GemmProblem* probs, int n, cudaStream_t stream) {
+  if (n < 0 || (n > 0 && probs == nullptr)) return KVP_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    const int rc = check_problem(probs[i]);
+    if (rc != KVP_OK) return rc;
+  }
+  // as many problems per launch as the parameter block holds
+  int begin = 0;
+  while (begin < n) {
+    int end = begin, maps = 0;
+    while (end < n && end - begin < MAX_PROB && maps + 2 * probs[end].nseg <= MAX_MAPS) maps += 2 * probs[end++].nseg;
+    const int rc = launch_group(probs + begin, end - begin, stream, 0, 0);
+    if (rc != KVP_OK) return rc;
+    begin = end;
+  }
+  return KVP_OK;
+}
+
+int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32,
+              cudaStream_t stream, int withhold_at, unsigned long long wait_limit_ns) {
+  if (nseg < 1 || nseg > MAX_SEG || segs == nullptr) return KVP_ERR_INVALID_ARG;
+  GemmProblem g{};
+  g.M = M;
+  g.N = N;
+  g.nseg = nseg;
+  for (int s = 0; s < nseg; ++s) g.segs[s] = segs[s];
+  g.a_mn = a_mn;
+  g.b_mn = b_mn;
+  g.c = c;
+  g.ldc = ldc;
+  g.out_f32 = out_f32;
+  const int rc = check_problem(g);
+  if (rc != KVP_OK) return rc;
+  return launch_group(&g, 1, stream, withhold_at, wait_limit_ns);
 }
 
 }  // namespace kvp

@@ -35,6 +35,21 @@ struct GemmSeg {
 int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32,
               cudaStream_t stream, int withhold_at = 0, unsigned long long wait_limit_ns = 0);
 
+// One problem of a grouped launch: C[M,N] = sum over segments, with its own operand modes and output type.
+struct GemmProblem {
+  int M, N;
+  GemmSeg segs[3];
+  int nseg;
+  int a_mn, b_mn;
+  void* c;
+  int64_t ldc;
+  int out_f32;
+};
+
+// All problems in as few launches as the kernel's parameter block allows (32 problems and 48 segments per launch);
+// the tiles are walked in the order of the list, so the problems with the longest tiles should come first.
+int gemm_grouped(const GemmProblem* probs, int n, cudaStream_t stream);
+
 int gemm_read_status();
 int attn_fwd_read_status();
 int attn_bwd_read_status();

@@ -420,6 +420,40 @@ def test_projection_backward_layer_by_layer_equals_one_call(kvp):
     assert kvp.device_status() == kvp.OK
 
 
+def test_projections_of_thirteen_layers_span_several_grouped_launches(kvp):
+    """Thirteen layers with eleven owners are 35 forward projections and 13 + 22 + 13 gradient GEMMs: more than one
+    grouped launch holds (32 problems; the backward takes eight layers at a time), with ragged M, N and K tiles in
+    every problem (T = 200, D = 192, Nq = 192, Nkv = 64)."""
+    donor = [0, 1, 1, 3, 4, 5, 6, 6, 8, 9, 10, 11, 12]
+    cfg = W.TrainCfg("thirteen-layers", 13, 2, 100, 192, 3, 1, 64, donor)
+    t = W.make_train_inputs(cfg, "cuda")
+    out = W.alloc_train_outputs(cfg, "cuda")
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+    kvp.proj_fwd(sh, donor, t["x"], t["wq"], t["wk"], t["wv"], out["q"], out["k"], out["v"])
+    g = torch.Generator(device="cpu").manual_seed(5)
+    dq = [(torch.randn(cfg.T, cfg.Hq * cfg.dh, generator=g) * 0.5).to(torch.bfloat16).cuda() for _ in range(cfg.L)]
+    dks = [None if donor[l] != l else (torch.randn(cfg.T, cfg.Hkv * cfg.dh, generator=g) * 0.5).cuda() for l in range(cfg.L)]
+    dvs = [None if donor[l] != l else (torch.randn(cfg.T, cfg.Hkv * cfg.dh, generator=g) * 0.5).cuda() for l in range(cfg.L)]
+    ws = torch.empty(kvp.workspace_bytes(kvp.OP_PROJ_BWD, sh, donor), dtype=torch.uint8, device="cuda")
+    kvp.proj_bwd(sh, donor, t["x"], t["wq"], t["wk"], t["wv"], dq, dks, dvs, out["dwq"], out["dwk"], out["dwv"],
+                 out["dx"], ws)
+    torch.cuda.synchronize()
+    assert kvp.device_status() == kvp.OK
+    x, wq, wk, wv = (f64l(t[n]) for n in ("x", "wq", "wk", "wv"))
+    q, k, v = A.proj_fwd(x, wq, wk, wv, donor, cfg.B, cfg.S, cfg.Hq, cfg.Hkv, cfg.dh)
+    rb = lambda a: None if a is None else A.round_bf16(f64(a))
+    dwq, dwk, dwv, dx = A.proj_bwd(x, wq, wk, wv, f64l(dq), [rb(a) for a in dks], [rb(a) for a in dvs], donor)
+    for l in range(cfg.L):
+        close(f"q[{l}]", out["q"][l], q[l])
+        close(f"dwq[{l}]", out["dwq"][l], dwq[l], sum_over_tokens=True)
+        close(f"dx[{l}]", out["dx"][l], dx[l])
+        if donor[l] == l:
+            close(f"k[{l}]", out["k"][l], k[l])
+            close(f"v[{l}]", out["v"][l], v[l])
+            close(f"dwk[{l}]", out["dwk"][l], dwk[l], sum_over_tokens=True)
+            close(f"dwv[{l}]", out["dwv"][l], dwv[l], sum_over_tokens=True)
+
+
 def test_c0_with_fp32_buffers(kvp):
     """The tiny stack with fp32 tensors in the caller's memory (dtype F32): forward, backward and decode steps.
     The library rounds fp32 inputs to bf16 on load and widens its bf16 results on store, so (i) every output

@@ -41,7 +41,10 @@ def test_workspace_queries_and_argument_validation_without_gpu(kvp):
     ws = kvp.workspace_bytes(kvp.OP_ATTN_BWD, sh, donor)
     # Delta [B,Hq,S] fp32 per layer + fp32 dQ accumulators for the member layers of one launch (at most 8)
     assert ws == 8 * (2 * 32 * 8192 * 4) + 8 * (2 * 32 * 8192 * 128 * 4)
-    assert kvp.workspace_bytes(kvp.OP_PROJ_BWD, sh, donor) == 2 * (2 * 8192 * 8 * 128 * 2)
+    # bf16 copies of the fp32 dK / dV sums of the owners of one grouped launch (5 owners here, at most 8)
+    assert kvp.workspace_bytes(kvp.OP_PROJ_BWD, sh, donor) == 5 * 2 * (2 * 8192 * 8 * 128 * 2)
+    assert kvp.workspace_bytes(kvp.OP_PROJ_BWD, kvp.Shape(12, 2, 8192, 4096, 32, 8, 128), list(range(12))) \
+        == 8 * 2 * (2 * 8192 * 8 * 128 * 2)
     assert kvp.workspace_bytes(kvp.OP_ATTN_FWD, sh, donor) == 0
     assert kvp.workspace_bytes(kvp.OP_ATTN_BWD, sh, [0, 0, 1, 0, 0, 0, 0, 0]) == 0   # invalid donor chain
     # entry points validate before touching the device

@@ -984,6 +984,9 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the shortened prefill and tail-stage runs of the default line")
     ap.add_argument("--no-e2e", action="store_true",
                     help="skip the end-to-end arms and the extra decode modes (for profiler launch lists: fewer launches)")
+    ap.add_argument("--gemm-pair-mode", type=int, default=1, choices=[0, 1, 2],
+                    help="GEMM tiles: 1 = CTA pairs for the forward GEMMs (the library's default), 0 = single-CTA tiles "
+                         "everywhere, 2 = CTA pairs everywhere (for comparison)")
     ap.add_argument("--small", action="store_true",
                     help="reduced shapes of the same kernels (inputs still larger than L2, under 2 GB on the device) "
                          "for profiler captures; implies --no-decode for train and --no-cpu-baseline")
@@ -1003,6 +1006,7 @@ def main():
     kdist.init("nccl")
     from paper_2608_15943_b200 import kvp     # loads the CUDA library or raises
     peaks, peaks_kind = measured_peaks()
+    kvp.set_gemm_pair_mode(args.gemm_pair_mode)
 
     if args.workload in ("train", "prefill"):
         line, cfg, backward = run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind)

@@ -71,6 +71,11 @@ int kvp_device_status(void);
  * (once: the word is cleared) and the device and the library remain usable.  Nothing faults and nothing spins
  * without a limit.  scratch: DEVICE memory, 16-byte aligned, at least 512 KiB, contents irrelevant and clobbered. */
 int kvp_selftest_bounded_wait(void* scratch, size_t scratch_bytes, kvp_stream_t stream);
+/* The same self-test on the CTA-pair GEMM kernel (one 256 x 256 tile on a cluster of two CTAs): the issuing CTA
+ * withholds, once, the arrivals that free a ring stage in both CTAs; both producers' waits run out, every role of
+ * both CTAs falls through to the common teardown (the two CTAs wait for each other, then free their TMEM).
+ * scratch: at least 768 KiB.  Refused with KVP_ERR_UNSUPPORTED while kvp_set_gemm_pair_mode(0) is in force. */
+int kvp_selftest_bounded_wait_pair(void* scratch, size_t scratch_bytes, kvp_stream_t stream);
 
 /* Benchmark bookkeeping.  kvp_launch_count: kernels launched by this library since it was loaded.
  * kvp_set_timing_events: record the caller's CUDA events (HOST arrays of n cudaEvent_t, created by
@@ -80,6 +85,12 @@ int kvp_selftest_bounded_wait(void* scratch, size_t scratch_bytes, kvp_stream_t 
 unsigned long long kvp_launch_count(void);
 int kvp_set_timing_events(int kernel, void** starts, void** stops, int n);
 int kvp_timing_events_used(int kernel);
+/* Measurement switch of the GEMM's tile shape.  1 (the default): the forward GEMMs (kvp_proj_fwd,
+ * kvp_out_proj_fwd, kvp_gemm) run on CTA pairs (256 x 256 tiles, one per pair of SMs) when every problem of the
+ * launch has more than 128 rows, the gradient GEMMs on single-CTA 128 x 256 tiles; 0: single-CTA tiles
+ * everywhere; 2: CTA pairs everywhere.  The results are the same in every mode (same products, same summation
+ * order along K).  Not thread-safe. */
+void kvp_set_gemm_pair_mode(int mode);
 
 /* ------------------------------------------------------------------------------------------
  * Planner (host only, pure, exact integer arithmetic).

@@ -228,7 +228,7 @@ extern "C" int kvp_proj_fwd(const kvp_shape* s, const int32_t* donor, const void
     probs.push_back(problem(T, Nkv, {x[l], wk[l], D, D, D}, 0, 0, k[l], Nkv, 0));
     probs.push_back(problem(T, Nkv, {x[l], wv[l], D, D, D}, 0, 0, v[l], Nkv, 0));
   }
-  return gemm_grouped(probs.data(), int(probs.size()), stream);
+  return gemm_grouped(probs.data(), int(probs.size()), stream, true);
 }
 
 extern "C" int kvp_proj_bwd(const kvp_shape* s, const int32_t* donor, const void* const* x, const void* const* wq,
@@ -316,7 +316,7 @@ extern "C" int kvp_proj_bwd_range(const kvp_shape* s, const int32_t* donor, cons
     }
     for (int l = c0; l < c1; ++l)
       if (donor[l] != l) probs.push_back(problem(T, D, {dq[l], wq[l], Nq, D, Nq}, 0, 1, dx[l], D, 0));
-    rc = gemm_grouped(probs.data(), int(probs.size()), stream);
+    rc = gemm_grouped(probs.data(), int(probs.size()), stream, false);
     if (rc != KVP_OK) return rc;
   }
   return KVP_OK;
@@ -335,7 +335,7 @@ extern "C" int kvp_out_proj_fwd(const kvp_shape* s, const void* const* o, const 
     if (o[l] == nullptr || wo[l] == nullptr || y[l] == nullptr) return KVP_ERR_INVALID_ARG;
     probs.push_back(problem(T, D, {o[l], wo[l], Nq, Nq, Nq}, 0, 0, y[l], D, 0));
   }
-  return gemm_grouped(probs.data(), int(probs.size()), stream);
+  return gemm_grouped(probs.data(), int(probs.size()), stream, true);
 }
 
 extern "C" int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const void* const* wo,
@@ -354,7 +354,7 @@ extern "C" int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const 
   for (int l = 0; l < s->L; ++l) probs.push_back(problem(D, Nq, {dy[l], o[l], D, Nq, T}, 1, 1, dwo[l], Nq, 1));
   // dO = dY Wo : A = dY [T, D] K-major, B = Wo stored [D, Nq] = [K, N] (MN-major)
   for (int l = 0; l < s->L; ++l) probs.push_back(problem(T, Nq, {dy[l], wo[l], D, Nq, D}, 0, 1, d_o[l], Nq, 0));
-  return gemm_grouped(probs.data(), int(probs.size()), stream);
+  return gemm_grouped(probs.data(), int(probs.size()), stream, false);
 }
 
 extern "C" int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,

@@ -138,6 +138,8 @@ extern "C" int kvp_timing_events_used(int kernel) {
   return kvp::g_timing[kernel].used;
 }
 
+extern "C" void kvp_set_gemm_pair_mode(int mode) { kvp::gemm_set_pair_mode(mode < 0 ? 0 : mode > 2 ? 2 : mode); }
+
 extern "C" int kvp_gemm(int M, int N, int K, const void* a, int64_t lda, int a_mn, const void* b, int64_t ldb,
                         int b_mn, void* c, int64_t ldc, int out_f32, kvp_stream_t stream) {
   kvp::GemmSeg seg{a, b, lda, ldb, K};
@@ -155,4 +157,17 @@ extern "C" int kvp_selftest_bounded_wait(void* scratch, size_t scratch_bytes, kv
   // producer's wait for that stage runs out after 5 ms
   return kvp::gemm_bf16(128, 256, &seg, 1, 0, 0, base + a_bytes + b_bytes, 256, 1, reinterpret_cast<cudaStream_t>(stream), 1,
                         5000000ull);
+}
+
+extern "C" int kvp_selftest_bounded_wait_pair(void* scratch, size_t scratch_bytes, kvp_stream_t stream) {
+  // A [256, 512] and B [256, 512] bf16, C [256, 256] fp32: one tile of the CTA-pair kernel
+  const size_t a_bytes = 256 * 512 * 2, b_bytes = 256 * 512 * 2, c_bytes = 256 * 256 * 4;
+  if (scratch == nullptr || scratch_bytes < a_bytes + b_bytes + c_bytes || !kvp::aligned16(scratch)) return KVP_ERR_WORKSPACE;
+  uint8_t* base = reinterpret_cast<uint8_t*>(scratch);
+  kvp::GemmSeg seg{base, base + a_bytes, 512, 512, 512};
+  // eight k-blocks through a six-stage ring: the arrivals that free the first stage in both CTAs are withheld, so
+  // both producers' waits for that stage run out after 5 ms
+  if (kvp::gemm_pair_mode() == 0) return KVP_ERR_UNSUPPORTED;
+  return kvp::gemm_bf16(256, 256, &seg, 1, 0, 0, base + a_bytes + b_bytes, 256, 1, reinterpret_cast<cudaStream_t>(stream), 1,
+                        5000000ull, true);
 }

@@ -32,8 +32,9 @@ struct GemmSeg {
 //   b_mn == 0: B_s stored [N, K] row-major (K-major);  b_mn == 1: stored [K, N] row-major.
 //   out_f32: C is fp32 (else bf16); ldc in elements.
 // withhold_at / wait_limit_ns serve the self-test of the bounded waits (kvp_selftest_bounded_wait) only.
+// prefer_pair: run on CTA pairs (256 x 256 tiles) when M > 128 and the pair mode allows it.
 int gemm_bf16(int M, int N, const GemmSeg* segs, int nseg, int a_mn, int b_mn, void* c, int64_t ldc, int out_f32,
-              cudaStream_t stream, int withhold_at = 0, unsigned long long wait_limit_ns = 0);
+              cudaStream_t stream, int withhold_at = 0, unsigned long long wait_limit_ns = 0, bool prefer_pair = true);
 
 // One problem of a grouped launch: C[M,N] = sum over segments, with its own operand modes and output type.
 struct GemmProblem {
@@ -48,8 +49,13 @@ struct GemmProblem {
 
 // All problems in as few launches as the kernel's parameter block allows (32 problems and 48 segments per launch);
 // the tiles are walked in the order of the list, so the problems with the longest tiles should come first.
-int gemm_grouped(const GemmProblem* probs, int n, cudaStream_t stream);
+// prefer_pair: CTA-pair tiles for this group (taken when every problem has more than 128 rows and the pair mode
+// allows it).  The forward projections ask for pairs; the gradient GEMMs of a training step do not: under the
+// board's power limit the attention backward sharing the step with them slowed by more than the pairs gained.
+int gemm_grouped(const GemmProblem* probs, int n, cudaStream_t stream, bool prefer_pair);
 
+void gemm_set_pair_mode(int mode);   // 0: single-CTA tiles only, 1: pairs where the caller prefers them, 2: pairs everywhere
+int gemm_pair_mode();
 int gemm_read_status();
 int attn_fwd_read_status();
 int attn_bwd_read_status();

@@ -242,6 +242,76 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar, uint32_t leader) {
 }
 
 // ----------------------------------------------------------------------------------------
+// CTA pairs (cta_group::2): two CTAs of one cluster, ranks 2i and 2i+1, whose tensor cores run one MMA with
+// M = 256 together.  Each CTA stages its own half of A and of B in its own shared memory and holds its own 128
+// rows of the accumulator in its own TMEM; the even CTA issues the MMAs for both.  Addresses of the partner's
+// barriers are shared::cluster addresses obtained with mapa.
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_addr_of(const void* local_smem, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(local_smem)), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are counted on a barrier of either CTA of the pair.
+__device__ __forceinline__ void tma_load_2d_pair_e(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y,
+                                                   uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred q;\n"
+      " setp.ne.b32 q, %5, 0;\n"
+      " @q cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+      "}\n" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(leader)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A[smem of both] * B[smem of both]; the descriptors name the same offsets in both CTAs.
+__device__ __forceinline__ void umma_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate, uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred p, q;\n"
+      " setp.ne.b32 p, %4, 0;\n"
+      " setp.ne.b32 q, %5, 0;\n"
+      " @q tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
+      : "memory");
+}
+// The barrier (of either CTA of the pair) receives one arrival once all pair MMAs issued so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr, uint32_t leader) {
+  asm volatile(
+      "{\n"
+      " .reg .pred q;\n"
+      " setp.ne.b32 q, %1, 0;\n"
+      " @q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+      "}\n" ::"r"(bar_cluster_addr),
+      "r"(leader)
+      : "memory");
+}
+
+// ----------------------------------------------------------------------------------------
 // TMEM <-> registers.  32x32b shape: thread i of the warp addresses lane (base + i); the warp
 // with (warp index % 4) == w may only touch lanes 32w .. 32w+31.
 // ----------------------------------------------------------------------------------------

@@ -25,7 +25,7 @@ PLACE_ARCH_BALANCED, PLACE_UNIFORM, PLACE_BIPOLAR = range(3)
 OP_PROJ_FWD, OP_PROJ_BWD, OP_ATTN_FWD, OP_ATTN_BWD, OP_DECODE = range(5)
 BF16, F32 = 0, 1   # dtype of the activations / weights in the caller's memory (kvp_shape.dtype, kvp_decode_desc.dtype)
 
-EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events",
+EXPORTS = ["kvp_status_string", "kvp_device_status", "kvp_launch_count", "kvp_set_timing_events", "kvp_set_gemm_pair_mode", "kvp_selftest_bounded_wait_pair",
            "kvp_timing_events_used", "kvp_plan", "kvp_layer_flops", "kvp_sim_1f1b", "kvp_workspace_bytes",
            "kvp_proj_fwd", "kvp_proj_bwd", "kvp_proj_bwd_range", "kvp_out_proj_fwd", "kvp_out_proj_bwd", "kvp_attn_fwd", "kvp_attn_bwd",
            "kvp_gemm", "kvp_rmsnorm", "kvp_rope", "kvp_swiglu", "kvp_add", "kvp_decode_workspace_bytes", "kvp_cache_append",
@@ -356,6 +356,16 @@ def launch_count() -> int:
     return int(lib.kvp_launch_count())
 
 
+lib.kvp_set_gemm_pair_mode.restype = None
+lib.kvp_set_gemm_pair_mode.argtypes = [C.c_int]
+
+
+def set_gemm_pair_mode(mode: int) -> None:
+    """kvp_set_gemm_pair_mode: 1 = CTA-pair tiles for the forward GEMMs (default), 0 = single-CTA tiles everywhere,
+    2 = CTA pairs everywhere."""
+    lib.kvp_set_gemm_pair_mode(int(mode))
+
+
 class KernelTimer:
     """Records CUDA events around up to n launches of one of the library's kernels and returns the
     per-launch durations in milliseconds."""
@@ -385,6 +395,16 @@ class KernelTimer:
 
 lib.kvp_selftest_bounded_wait.restype = C.c_int
 lib.kvp_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+lib.kvp_selftest_bounded_wait_pair.restype = C.c_int
+lib.kvp_selftest_bounded_wait_pair.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+def selftest_bounded_wait_pair(scratch: torch.Tensor):
+    """kvp_selftest_bounded_wait_pair: the same self-test on the CTA-pair GEMM kernel (scratch of at least 768 KiB)."""
+    _check(lib.kvp_selftest_bounded_wait_pair(scratch.data_ptr(), scratch.numel() * scratch.element_size(), _stream()),
+           "kvp_selftest_bounded_wait_pair")
 
 
 def selftest_bounded_wait(scratch: torch.Tensor):

@@ -99,6 +99,50 @@ def test_gemm_all_layouts(kvp, M, N, K, a_mn, b_mn):
     assert kvp.device_status() == kvp.OK
 
 
+@pytest.mark.parametrize("M,N,K", [(264, 8, 8), (304, 520, 200), (1280, 768, 1096)])
+@pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 0), (1, 1)])
+def test_gemm_on_cta_pairs_equals_single_cta_tiles(kvp, M, N, K, a_mn, b_mn):
+    """The 256 x 256 tiles of the CTA-pair kernel and the 128 x 256 tiles of the single-CTA kernel sum the same
+    products in the same order along K: bit-identical outputs, also with ragged last tiles in M, N and K (and a
+    second half-tile that lies entirely outside M)."""
+    a = synth.normal((M, K), 13, 1, 1.0, "cuda")
+    b = synth.normal((N, K), 13, 2, 1.0, "cuda")
+    sa = a.t().contiguous() if a_mn else a
+    sb = b.t().contiguous() if b_mn else b
+    out = {}
+    try:
+        for mode in (0, 2):
+            kvp.set_gemm_pair_mode(mode)
+            gd = Guarded()
+            out[mode] = gd.empty((M, N), torch.float32, float("nan"))
+            kvp.gemm(sa, sb, out[mode], a_mn, b_mn)
+            gd.check()
+    finally:
+        kvp.set_gemm_pair_mode(1)
+    assert torch.equal(out[0], out[2])
+    close("gemm on pairs", out[2], f64(a) @ f64(b).T, rel=1e-5, abs_=1e-4, sum_over_tokens=True)
+    assert kvp.device_status() == kvp.OK
+
+
+def test_bounded_wait_runs_out_cleanly_on_a_cta_pair(kvp):
+    """The same failure detection on the CTA-pair GEMM kernel: the issuing CTA withholds the arrivals that free a
+    ring stage in both CTAs of the cluster; both give up after 5 ms, wait for each other, free their TMEM and exit."""
+    assert kvp.device_status() == kvp.OK
+    scratch = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    kvp.selftest_bounded_wait_pair(scratch)
+    assert kvp.device_status() == kvp.ERR_TIMEOUT
+    assert kvp.device_status() == kvp.OK
+    with pytest.raises(kvp.KvpError) as e:
+        kvp.selftest_bounded_wait_pair(scratch[:512 * 1024])
+    assert e.value.status == kvp.ERR_WORKSPACE
+    a = synth.normal((512, 512), 9, 1, 1.0, "cuda")
+    b = synth.normal((384, 512), 9, 2, 1.0, "cuda")
+    c = torch.full((512, 384), float("nan"), device="cuda")
+    kvp.gemm(a, b, c, 0, 0)                              # runs on CTA pairs again
+    close("pair gemm after a timed-out launch", c, f64(a) @ f64(b).T, rel=1e-5, abs_=1e-4, sum_over_tokens=True)
+    assert kvp.device_status() == kvp.OK
+
+
 def test_bounded_wait_runs_out_cleanly_and_the_library_stays_usable(kvp):
     """Failure detection on the device: a wait that nothing satisfies gives up after its limit, the kernel
     records the timeout, frees its TMEM and exits; the host reads the status and carries on.  The library's

@@ -4,13 +4,20 @@
 // One CTA owns TWO adjacent 128-row query tiles (A, B) of one (batch, query head) and walks the
 // donor's K/V tiles once for both, so every K/V tile fetched by TMA feeds twice the tensor work.
 //   warp 0      TMA producer: Q_A, Q_B once, then K_j / V_j rings
-//   warp 1      tcgen05.mma issuer: S_X = Q_X K_j^T into tile X's 128 TMEM columns, and
-//               O_X += P_X V_j with P_X as the A operand FROM TMEM (bf16 pairs written back over the
-//               first 64 columns of S_X) and V_j as an MN-major B operand
-//   warps 2-5   softmax of tile A, warps 6-9 softmax of tile B: one thread per query row (TMEM lane
+//   warps 1, 2  tcgen05.mma issuers, one per query tile (on two different warp schedulers: issuing an MMA costs
+//               its scheduler some tens of cycles, which the softmax warps of that scheduler would otherwise
+//               have).  Every 128-key tile is worked on as two 64-key sub-blocks c = 2j, 2j+1:
+//               S_X(c) = Q_X K_c^T goes into one of TWO 64-column score buffers of tile X (c & 1), and
+//               O_X += P_X(c) V_c takes P_X(c) as the A operand FROM TMEM (bf16 pairs written back over the
+//               first 32 columns of that score buffer) and V_c as an MN-major B operand.  S_X(c+2) is issued
+//               right behind P_X(c) V_c, so the scores of sub-block c+1 are already complete when the softmax
+//               of sub-block c ends: the softmax warps never wait for the tensor pipe to turn around.
+//   warp 3      idle
+//   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one thread per query row (TMEM lane
 //               == row, so the row maximum and sum need no cross-thread traffic), packed fp32x2
-//               arithmetic, O rescaled in TMEM only when the running maximum moved by more than 2^8
-// While one tile's exponentials run, the tensor pipe works on the other tile.
+//               arithmetic, O rescaled in TMEM only when the running maximum moved by more than 2^8 (and
+//               then only after the P V product still in flight has completed)
+// While one tile's exponentials run, the tensor pipe works on the other tile and on the next scores of this one.
 #include <math.h>
 
 #include "kvp_host.h"
@@ -20,7 +27,8 @@ namespace kvp {
 namespace {
 
 constexpr int BQ = 128, BKV = 128;
-constexpr int FWD_THREADS = 320;
+constexpr int BC = 64;            // keys per sub-block (one score buffer)
+constexpr int FWD_THREADS = 384;
 constexpr int FWD_KSTAGES = 3;
 constexpr int FWD_VSTAGES = 2;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
@@ -58,7 +66,6 @@ template <int DH>
 __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_constant__ FwdParams p) {
   using L = FwdSmem<DH>;
   constexpr int KSTEPS_QK = DH / 16;   // K dimension of S = Q K^T is dh
-  constexpr int KSTEPS_PV = BKV / 16;  // K dimension of O = P V is the kv tile
   constexpr int HALVES = DH / 64;      // 64-column (128-byte) blocks per row of Q / K / V
 
   extern __shared__ uint8_t smem_raw[];
@@ -69,9 +76,10 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
   uint64_t* k_empty = k_full + FWD_KSTAGES;     // [KSTAGES]
   uint64_t* v_full = k_empty + FWD_KSTAGES;     // [VSTAGES]
   uint64_t* v_empty = v_full + FWD_VSTAGES;     // [VSTAGES]
-  uint64_t* s_full = v_empty + FWD_VSTAGES;     // [2] per query tile
-  uint64_t* p_ready = s_full + 2;               // [2] per query tile (128 arrivals)
-  uint64_t* o_done = p_ready + 2;               // [2] per query tile
+  uint64_t* s_full = v_empty + FWD_VSTAGES;     // [2][2] per query tile and score buffer
+  uint64_t* p_ready = s_full + 4;               // [2][2] per query tile and score buffer (128 arrivals)
+  uint64_t* pv_done = p_ready + 4;              // [2] per query tile: one completion per sub-block's P V product
+  uint64_t* o_done = pv_done + 2;               // [2] per query tile
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_done + 2);
 
   const int warp = threadIdx.x >> 5;
@@ -99,15 +107,18 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
     mbar_init(q_full, 1);
     for (int i = 0; i < FWD_KSTAGES; ++i) {
       mbar_init(&k_full[i], 1);
-      mbar_init(&k_empty[i], 1);
+      mbar_init(&k_empty[i], 2);   // one MMA-completion arrival per issuing warp
     }
     for (int i = 0; i < FWD_VSTAGES; ++i) {
       mbar_init(&v_full[i], 1);
-      mbar_init(&v_empty[i], 1);
+      mbar_init(&v_empty[i], 2);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 4; ++i) {
       mbar_init(&s_full[i], 1);
       mbar_init(&p_ready[i], 128);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&pv_done[i], 1);
       mbar_init(&o_done[i], 1);
     }
     mbar_fence_init();
@@ -120,7 +131,8 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // tile X: scores / P at [X*128, X*128+128), output accumulator at [256 + X*128, ...)
+  // tile X: score buffer u at [X*128 + u*64, +64) with P over its first 32 columns; output accumulator at
+  // [256 + X*128, +128)
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -159,66 +171,76 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         if (ok) ok = load_v(j);
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------ MMA issuer of query tile x ------------------------------
     {
       const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
-      constexpr uint32_t idesc_qk = umma_idesc_bf16(BQ, BKV, 0, 0);
+      constexpr uint32_t idesc_qk = umma_idesc_bf16(BQ, BC, 0, 0);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(BQ, DH, 0, 1);
       constexpr uint32_t hi = desc_hi_sw128(1024);
+      constexpr int KSTEPS_SUB = BC / 16;  // K steps of one sub-block's P V product
       const uint32_t k_base = smem_u32(smem + L::OFF_K), v_base = smem_u32(smem + L::OFF_V);
+      const int x = warp - 1;
+      const int n_cx = 2 * n_kv[x];
+      const int n_cmax = 2 * n_max;
       bool ok = mbar_wait(q_full, 0, err);
-      auto issue_s = [&](int x, int j) {  // S_x(j) = Q_x K_j^T; K_j is known to be resident
-        const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q + x * L::Q_BYTES), 0);
-        const uint32_t k_lo = desc_lo_sw128(k_base + (j % FWD_KSTAGES) * L::KV_BYTES, 0);
+      const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::OFF_Q + x * L::Q_BYTES), 0);
+      const uint32_t tm_sx = tmem_base + x * BKV, tm_ox = tmem_base + 256 + x * 128;
+      auto issue_s = [&](int c) {  // S_x(c) = Q_x K_c^T; the key tile holding sub-block c is known to be resident
+        const int j = c >> 1, u = c & 1;
+        // keys 64u .. 64u+63 of the tile are rows 64u .. of each 128-byte-wide block: 64 rows x 128 B further on
+        const uint32_t k_lo = desc_lo_sw128(k_base + (j % FWD_KSTAGES) * L::KV_BYTES + u * (BC * 128), 0);
 #pragma unroll
         for (int ks = 0; ks < KSTEPS_QK; ++ks) {
           const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-          umma_ss_w(tmem_base + x * BKV, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0, leader);
+          umma_ss_w(tm_sx + u * BC, desc_lo_add(q_lo, off), desc_lo_add(k_lo, off), hi, idesc_qk, ks != 0, leader);
         }
-        umma_commit(&s_full[x], leader);
+        umma_commit(&s_full[2 * x + u], leader);
       };
-      auto issue_pv = [&](int x, int j) {  // O_x += P_x(j) V_j
+      auto issue_pv = [&](int c) {  // O_x += P_x(c) V_c
+        const int j = c >> 1, u = c & 1;
         const uint32_t v_lo = desc_lo_sw128(v_base + (j % FWD_VSTAGES) * L::KV_BYTES, HALF_BYTES);
 #pragma unroll
-        for (int ks = 0; ks < KSTEPS_PV; ++ks)
-          umma_ts_w(tmem_base + 256 + x * 128, tmem_base + x * BKV + ks * 8, desc_lo_add(v_lo, ks * 2048), hi, idesc_pv,
-                    (j | ks) != 0, leader);
+        for (int ks = 0; ks < KSTEPS_SUB; ++ks)
+          umma_ts_w(tm_ox, tm_sx + u * BC + ks * 8, desc_lo_add(v_lo, (u * KSTEPS_SUB + ks) * 2048), hi, idesc_pv,
+                    (c | ks) != 0, leader);
       };
       if (ok && n_max > 0) {
         ok = mbar_wait(&k_full[0], 0, err);
         if (ok) {
           tc_fence_after_sync();
-          if (n_kv[0] > 0) issue_s(0, 0);
-          if (n_kv[1] > 0) issue_s(1, 0);
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+            if (c < n_cx) issue_s(c);
           umma_commit(&k_empty[0], leader);
         }
       }
-      for (int j = 0; j < n_max && ok; ++j) {
-        const bool next = j + 1 < n_max;
-        if (next) {
-          if (!mbar_wait(&k_full[(j + 1) % FWD_KSTAGES], ((j + 1) / FWD_KSTAGES) & 1, err)) { ok = false; break; }
+      // Every round releases its K / V stages from this warp too when this tile has run out of sub-blocks (the
+      // other tile may be one key tile longer): an arrival with nothing outstanding completes at once.
+      for (int c = 0; c < n_cmax && ok; ++c) {
+        const int j = c >> 1, u = c & 1;
+        const int cn = c + 2, jn = cn >> 1;   // the scores issued in this round: sub-block c + 2
+        // (it still waits for every stage to fill first, so it can never arrive twice in one phase of a stage)
+        if (u == 0 && !mbar_wait(&v_full[j % FWD_VSTAGES], (j / FWD_VSTAGES) & 1, err)) { ok = false; break; }
+        if (cn < n_cmax && (cn & 1) == 0) {
+          if (!mbar_wait(&k_full[jn % FWD_KSTAGES], (jn / FWD_KSTAGES) & 1, err)) { ok = false; break; }
         }
-        if (!mbar_wait(&v_full[j % FWD_VSTAGES], (j / FWD_VSTAGES) & 1, err)) { ok = false; break; }
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          if (j < n_kv[x]) {
-            if (!mbar_wait(&p_ready[x], j & 1, err)) { ok = false; break; }
-            tc_fence_after_sync();
-            issue_pv(x, j);
-            if (j + 1 == n_kv[x]) umma_commit(&o_done[x], leader);
-            // the score buffer of tile x is free again once P_x(j) V_j has been issued (in-order pipe)
-            if (j + 1 < n_kv[x]) issue_s(x, j + 1);
-          }
+        if (c < n_cx) {
+          if (!mbar_wait(&p_ready[2 * x + u], (c >> 1) & 1, err)) { ok = false; break; }
+          tc_fence_after_sync();
+          issue_pv(c);
+          umma_commit(&pv_done[x], leader);
+          if (c + 1 == n_cx) umma_commit(&o_done[x], leader);
+          // score buffer u is free again once P_x(c) V_c has been issued (in-order pipe, same issuing thread)
+          if (cn < n_cx) issue_s(cn);
         }
-        if (!ok) break;
-        umma_commit(&v_empty[j % FWD_VSTAGES], leader);
-        if (next) umma_commit(&k_empty[(j + 1) % FWD_KSTAGES], leader);
+        if (u == 1) umma_commit(&v_empty[j % FWD_VSTAGES], leader);
+        if (cn < n_cmax && (cn & 1) == 1) umma_commit(&k_empty[jn % FWD_KSTAGES], leader);
       }
     }
-  } else {
+  } else if (warp >= 4) {
     // ------------------------------ softmax + epilogue ------------------------------
-    const int x = (warp - 2) >> 2;      // query tile of this warpgroup
+    const int x = (warp - 4) >> 2;      // query tile of this warpgroup
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;  // row inside the query tile == TMEM lane
     const int q_row = q0 + x * BQ + r;
@@ -226,42 +248,43 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
     const uint32_t tm_s = tmem_base + x * BKV + lane_sel;
     const uint32_t tm_o = tmem_base + 256 + x * 128 + lane_sel;
     const int my_n = n_kv[x];
+    const int my_c = 2 * my_n;
     const uint64_t c2 = pack_f2(p.scale_log2, p.scale_log2);
     float m_used = -INFINITY;  // running maximum (log2 domain) the exponentials are taken against
     uint64_t l2 = 0ull, l2b = 0ull;  // four partial row sums (two packed pairs, for independent add chains)
     bool ok = true;
-    for (int j = 0; j < my_n; ++j) {
-      ok = mbar_wait(&s_full[x], j & 1, err);
+    for (int c = 0; c < my_c; ++c) {
+      const int u = c & 1;
+      ok = mbar_wait(&s_full[2 * x + u], (c >> 1) & 1, err);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       tc_fence_after_sync();
-      uint32_t sv[BKV];  // raw scores of this row
-      tmem_ld_x32(tm_s, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-      tmem_ld_x32(tm_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
-      tmem_ld_x32(tm_s + 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[64]));
-      tmem_ld_x32(tm_s + 96, *reinterpret_cast<uint32_t(*)[32]>(&sv[96]));
+      const uint32_t tm_su = tm_s + u * BC;
+      uint32_t sv[BC];  // raw scores of this row
+      tmem_ld_x32(tm_su, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+      tmem_ld_x32(tm_su + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
       tmem_ld_wait();
-      // columns of this tile visible to this row
-      const int kv0 = j * BKV;
+      // columns of this sub-block visible to this row
+      const int kv0 = c * BC;
       int lim = p.S - kv0;
       if (p.causal) lim = min(lim, q_row - kv0 + 1);
-      if (__any_sync(0xffffffffu, lim < BKV)) {
+      if (__any_sync(0xffffffffu, lim < BC)) {
 #pragma unroll
-        for (int i = 0; i < BKV; ++i)
+        for (int i = 0; i < BC; ++i)
           if (i >= lim) sv[i] = 0xff800000u;  // -inf
       }
-      // four independent partial maxima: one 64-deep dependent chain would cost its full latency per tile
+      // four independent partial maxima: one long dependent chain would cost its full latency per sub-block
       float mp[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) mp[u] = fmaxf(__uint_as_float(sv[2 * u]), __uint_as_float(sv[2 * u + 1]));
+      for (int w = 0; w < 4; ++w) mp[w] = fmaxf(__uint_as_float(sv[2 * w]), __uint_as_float(sv[2 * w + 1]));
 #pragma unroll
-      for (int i = 8; i < BKV; i += 8)
+      for (int i = 8; i < BC; i += 8)
 #pragma unroll
-        for (int u = 0; u < 4; ++u) mp[u] = fmax3(mp[u], __uint_as_float(sv[i + 2 * u]), __uint_as_float(sv[i + 2 * u + 1]));
+        for (int w = 0; w < 4; ++w) mp[w] = fmax3(mp[w], __uint_as_float(sv[i + 2 * w]), __uint_as_float(sv[i + 2 * w + 1]));
       const float m_raw = fmaxf(fmaxf(mp[0], mp[1]), fmaxf(mp[2], mp[3]));
       const float m_tile = m_raw * p.scale_log2;  // the scale is positive, so the maximum commutes with it
       float alpha = 1.f;
       bool rescale = false;
-      if (j == 0) {
+      if (c == 0) {
         m_used = m_tile;
       } else if (m_tile > m_used + kRescaleThreshold) {
         alpha = fast_exp2(m_used - m_tile);
@@ -272,32 +295,36 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
       }
       const uint64_t nm2 = pack_f2(-m_used, -m_used);
 #pragma unroll
-      for (int c = 0; c < BKV / 32; ++c) {
+      for (int g = 0; g < BC / 32; ++g) {
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const uint64_t t = ffma2(pack_f2(__uint_as_float(sv[c * 32 + 2 * i]), __uint_as_float(sv[c * 32 + 2 * i + 1])), c2, nm2);
+          const uint64_t t = ffma2(pack_f2(__uint_as_float(sv[g * 32 + 2 * i]), __uint_as_float(sv[g * 32 + 2 * i + 1])), c2, nm2);
           const uint64_t e = pack_f2(fast_exp2(f2_lo(t)), fast_exp2(f2_hi(t)));
           if (i & 1) l2b = fadd2(l2b, e); else l2 = fadd2(l2, e);
           pk[i] = pack_bf16(f2_lo(e), f2_hi(e));
         }
-        tmem_st_x16(tm_s + c * 16, pk);  // P as bf16 pairs over the first 64 columns of the score buffer
+        tmem_st_x16(tm_su + g * 16, pk);  // P as bf16 pairs over the first 32 columns of this score buffer
       }
-      // O_x is idle here: P_x(j-1) V_{j-1} precedes S_x(j) in the in-order tensor pipe
-      if (j > 0 && __any_sync(0xffffffffu, rescale)) {
+      // O_x may still be receiving P_x(c-1) V_(c-1): a rescale waits for that product first.  P_x(c) V_c is not
+      // issued before this warpgroup's arrival below.
+      if (c > 0 && __any_sync(0xffffffffu, rescale)) {
+        bool w = mbar_wait(&pv_done[x], (c - 1) & 1, err);
+        if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+        tc_fence_after_sync();
 #pragma unroll
-        for (int c = 0; c < DH / 32; ++c) {
+        for (int g = 0; g < DH / 32; ++g) {
           uint32_t tmp[32];
-          tmem_ld_x32(tm_o + c * 32, tmp);
+          tmem_ld_x32(tm_o + g * 32, tmp);
           tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; ++i) tmp[i] = __float_as_uint(__uint_as_float(tmp[i]) * alpha);
-          tmem_st_x32(tm_o + c * 32, tmp);
+          tmem_st_x32(tm_o + g * 32, tmp);
         }
       }
       tmem_st_wait();
       tc_fence_before_sync();
-      mbar_arrive(&p_ready[x]);
+      mbar_arrive(&p_ready[2 * x + u]);
     }
     ok = __all_sync(0xffffffffu, ok);
     if (ok && my_n > 0) {

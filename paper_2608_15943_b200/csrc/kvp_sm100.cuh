@@ -49,20 +49,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same test, but the hardware may park the thread until the phase completes or suspend_ns have passed: a
+// waiting warp then takes no issue slots from the warps that share its scheduler.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t suspend_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      " .reg .pred p;\n"
+      " mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      " selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(suspend_ns)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false after limit_ns, or as soon as another thread has flagged an
 // error; the caller must then leave its role loop and fall through to the common teardown.
+// Between two looks at the error flag and the clock the thread is parked on the barrier for up to
+// kParkNs, so a role that waits costs the other warps of its scheduler nothing.
+constexpr uint32_t kParkNs = 20000;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err,
                                           unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
-  uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if (((++spins) & 0xFF) == 0) {
-      if (*reinterpret_cast<volatile int*>(err) != 0) return false;
-      if (globaltimer_ns() - t0 > limit_ns) {
-        atomicExch(err, KVP_DEV_TIMEOUT);
-        return false;
-      }
+  while (!mbar_try_wait_parked(bar, parity, kParkNs)) {
+    if (*reinterpret_cast<volatile int*>(err) != 0) return false;
+    if (globaltimer_ns() - t0 > limit_ns) {
+      atomicExch(err, KVP_DEV_TIMEOUT);
+      return false;
     }
   }
   return true;

@@ -267,7 +267,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
       const int kv0 = c * BC;
       int lim = p.S - kv0;
       if (p.causal) lim = min(lim, q_row - kv0 + 1);
-      if (__any_sync(0xffffffffu, lim < BC)) {
+      // (no vote for the sub-blocks that every row of the tile sees in full: the common case)
+      const bool all_visible = kv0 + BC <= p.S && (!p.causal || kv0 + BC - 1 <= q0 + x * BQ);
+      if (!all_visible && __any_sync(0xffffffffu, lim < BC)) {
 #pragma unroll
         for (int i = 0; i < BC; ++i)
           if (i >= lim) sv[i] = 0xff800000u;  // -inf

@@ -1,5 +1,5 @@
 // Blackwell (sm_100a) primitives used by every kernel of the library: mbarrier with bounded
-// waits, TMA tensor copies (never multicast), tcgen05 MMA / TMEM, shared-memory matrix
+// waits, TMA tensor copies (every CTA issues its own loads), tcgen05 MMA / TMEM, shared-memory matrix
 // descriptors.  Inline PTX only; no third-party headers.
 #pragma once
 #include <cuda.h>

@@ -498,6 +498,51 @@ def test_projections_of_thirteen_layers_span_several_grouped_launches(kvp):
             close(f"dwv[{l}]", out["dwv"][l], dwv[l], sum_over_tokens=True)
 
 
+def test_projection_block_is_bit_identical_on_cta_pairs_and_single_cta_tiles(kvp):
+    """Every projection GEMM of a small block -- forward (K-major operands), weight gradients (both operands
+    MN-major, fp32 output, K = all tokens) and input gradients (three K segments into one tile) -- gives the same
+    bits on the CTA-pair kernel as on the single-CTA kernel.  All problems have more than 128 rows, so pair mode 2
+    really puts every grouped launch on pairs."""
+    donor = [0, 0, 2]
+    cfg = W.TrainCfg("pairs-vs-single", 3, 2, 200, 192, 4, 2, 128, donor)
+    t = W.make_train_inputs(cfg, "cuda")
+    sh = kvp.Shape(cfg.L, cfg.B, cfg.S, cfg.D, cfg.Hq, cfg.Hkv, cfg.dh)
+    g = torch.Generator(device="cpu").manual_seed(17)
+    dq = [(torch.randn(cfg.T, cfg.Hq * cfg.dh, generator=g) * 0.5).to(torch.bfloat16).cuda() for _ in range(cfg.L)]
+    dks = [None if donor[l] != l else (torch.randn(cfg.T, cfg.Hkv * cfg.dh, generator=g) * 0.5).cuda() for l in range(cfg.L)]
+    dvs = [None if donor[l] != l else (torch.randn(cfg.T, cfg.Hkv * cfg.dh, generator=g) * 0.5).cuda() for l in range(cfg.L)]
+    ws = torch.empty(kvp.workspace_bytes(kvp.OP_PROJ_BWD, sh, donor), dtype=torch.uint8, device="cuda")
+    outs = {}
+    try:
+        for mode in (0, 2):
+            kvp.set_gemm_pair_mode(mode)
+            out = W.alloc_train_outputs(cfg, "cuda")
+            for name in ("q", "k", "v", "dwq", "dwk", "dwv", "dx"):
+                for a in out[name]:
+                    if a is not None:
+                        a.fill_(float("nan"))
+            kvp.proj_fwd(sh, donor, t["x"], t["wq"], t["wk"], t["wv"], out["q"], out["k"], out["v"])
+            kvp.proj_bwd(sh, donor, t["x"], t["wq"], t["wk"], t["wv"], dq, dks, dvs, out["dwq"], out["dwk"], out["dwv"],
+                         out["dx"], ws)
+            torch.cuda.synchronize()
+            outs[mode] = out
+    finally:
+        kvp.set_gemm_pair_mode(1)
+    assert kvp.device_status() == kvp.OK
+    for name in ("q", "k", "v", "dwq", "dwk", "dwv", "dx"):
+        for l in range(cfg.L):
+            a, b = outs[0][name][l], outs[2][name][l]
+            if a is not None:
+                assert not torch.isnan(a.float()).any(), (name, l)
+                assert torch.equal(a, b), (name, l)
+    x, wq, wk, wv = (f64l(t[n]) for n in ("x", "wq", "wk", "wv"))
+    rb = lambda a: None if a is None else A.round_bf16(f64(a))
+    dwq, dwk, dwv, dx = A.proj_bwd(x, wq, wk, wv, f64l(dq), [rb(a) for a in dks], [rb(a) for a in dvs], donor)
+    for l in range(cfg.L):
+        close(f"dx[{l}] on pairs", outs[2]["dx"][l], dx[l])
+        close(f"dwq[{l}] on pairs", outs[2]["dwq"][l], dwq[l], sum_over_tokens=True)
+
+
 def test_c0_with_fp32_buffers(kvp):
     """The tiny stack with fp32 tensors in the caller's memory (dtype F32): forward, backward and decode steps.
     The library rounds fp32 inputs to bf16 on load and widens its bf16 results on store, so (i) every output

@@ -220,7 +220,7 @@ int kvp_out_proj_bwd(const kvp_shape* s, const void* const* o, const void* const
 
 /* Eq. 2-3.  o[l] = softmax(q[l] k[d]^T * scale + M) v[d] with d = donor[l], M the causal mask when
  * causal != 0 (key j visible to query i iff j <= i); scale == 0 means 1/sqrt(dh).
- * o[l]: [B,S,Hq,dh] bf16; lse[l]: [B,Hq,S] fp32. */
+ * o[l]: [B,S,Hq,dh] bf16; lse[l]: [B,Hq,S] fp32.  Up to eight layers run as one launch of persistent CTAs. */
 int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
                  const void* const* k, const void* const* v, void* const* o, float* const* lse, void* ws,
                  size_t ws_bytes, kvp_stream_t stream);

@@ -6,8 +6,9 @@
 #include "kvp_host.h"
 
 namespace kvp {
-int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, const void* k, const void* v, void* o,
-                   float* lse, cudaStream_t stream);
+int attn_fwd_layers(const kvp_shape* s, int causal, float scale, const void* const* q, const void* const* k,
+                    const void* const* v, void* const* o, float* const* lse, int n, cudaStream_t stream);
+int attn_fwd_max_layers();
 size_t attn_bwd_workspace(const kvp_shape* s, const int32_t* donor);
 int attn_bwd_all(const kvp_shape* s, const int32_t* donor, int causal, float scale, const void* const* q,
                  const void* const* k, const void* const* v, const void* const* o, const void* const* d_o,
@@ -382,9 +383,16 @@ extern "C" int kvp_attn_fwd(const kvp_shape* s, const int32_t* donor, int causal
     rc = kvp_attn_fwd(&s16, donor, causal, scale, q16, k16, v16, o16, lse, ws, ws_bytes, stream_);
     return rc != KVP_OK ? rc : sh.finish();
   }
+  // up to eight layers per launch, each with the K / V of its donor
+  std::vector<const void*> kd(size_t(s->L)), vd(size_t(s->L));
   for (int l = 0; l < s->L; ++l) {
-    const int d = donor[l];
-    rc = attn_fwd_layer(s, causal, scale, q[l], k[d], v[d], o[l], lse[l], stream);
+    kd[l] = k[donor[l]];
+    vd[l] = v[donor[l]];
+  }
+  const int chunk = attn_fwd_max_layers();
+  for (int l0 = 0; l0 < s->L; l0 += chunk) {
+    const int n = std::min(chunk, s->L - l0);
+    rc = attn_fwd_layers(s, causal, scale, q + l0, kd.data() + l0, vd.data() + l0, o + l0, lse + l0, n, stream);
     if (rc != KVP_OK) return rc;
   }
   return KVP_OK;

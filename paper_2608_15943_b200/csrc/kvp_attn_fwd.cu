@@ -48,10 +48,14 @@ struct FwdSmem {
   static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // + alignment slack
 };
 
+constexpr int FWD_MAX_LAYERS = 8;   // layers per launch
+
 struct FwdParams {
-  CUtensorMap map_q, map_k, map_v;  // 4-D [B, S, H, dh] tensors, box {64, 1, 128, 1}
-  __nv_bfloat16* o;                 // [B, S, Hq, dh]
-  float* lse;                       // [B, Hq, S]
+  // per layer: 4-D [B, S, H, dh] tensors, box {64, 1, 128, 1}; K and V are those of the layer's donor
+  CUtensorMap map_q[FWD_MAX_LAYERS], map_k[FWD_MAX_LAYERS], map_v[FWD_MAX_LAYERS];
+  __nv_bfloat16* o[FWD_MAX_LAYERS];  // [B, S, Hq, dh]
+  float* lse[FWD_MAX_LAYERS];        // [B, Hq, S]
+  int n_layers;
   int B, S, Hq, Hkv;
   int causal;
   float scale_log2;                 // scale * log2(e)
@@ -63,7 +67,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// Work items of a launch: (batch, query head, pair of query tiles), the deepest causal pairs first.  The list is
+// Work items of a launch: (layer, batch, query head, pair of query tiles), the deepest causal pairs first.  The list is
 // dealt out in rounds of gridDim.x items, forwards in even rounds and backwards in odd ones, so that the CTA that
 // got the longest item of one round gets the shortest of the next: every CTA ends up with nearly the same work.
 __device__ __forceinline__ int fwd_item_index(int round) {
@@ -71,17 +75,18 @@ __device__ __forceinline__ int fwd_item_index(int round) {
   return round * g + ((round & 1) ? g - 1 - i : i);
 }
 struct FwdItem {
-  int b, hq, hk, q0;
+  int layer, b, hq, hk, q0;
   int n_kv[2];  // key tiles each query tile walks (tile B may not exist at a ragged end)
   int n_max;
 };
 __device__ __forceinline__ FwdItem fwd_item(const FwdParams& p, int t, int n_pairs) {
   FwdItem w;
-  const int bh = p.B * p.Hq;
-  const int pair = n_pairs - 1 - t / bh;
-  const int r = t % bh;
+  const int bh = p.B * p.Hq, lbh = p.n_layers * bh;
+  const int pair = n_pairs - 1 - t / lbh;
+  const int r = t % lbh;
+  w.layer = r / bh;
   w.hq = r % p.Hq;
-  w.b = r / p.Hq;
+  w.b = (r % bh) / p.Hq;
   w.hk = w.hq / (p.Hq / p.Hkv);
   w.q0 = pair * 2 * BQ;  // first row of tile A; tile B starts at q0 + 128
 #pragma unroll
@@ -122,7 +127,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
 
   const int n_qtiles = (p.S + BQ - 1) / BQ;
   const int n_pairs = (n_qtiles + 1) / 2;
-  const int n_items = n_pairs * p.B * p.Hq;
+  const int n_items = n_pairs * p.n_layers * p.B * p.Hq;
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
@@ -167,9 +172,6 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
     // ------------------------------ TMA producer ------------------------------
     {
       const uint32_t leader = elect_one();  // the whole warp runs the loop; one lane issues
-      if (leader) tma_prefetch_desc(&p.map_q);
-      if (leader) tma_prefetch_desc(&p.map_k);
-      if (leader) tma_prefetch_desc(&p.map_v);
       uint32_t it = 0, kg = 0, vg = 0;  // items, K tiles and V tiles requested so far
       bool ok = true;
       for (int round = 0; round * int(gridDim.x) < n_items && ok; ++round) {
@@ -182,14 +184,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         for (int x = 0; x < 2; ++x)
 #pragma unroll
           for (int h = 0; h < HALVES; ++h)
-            tma_load_4d_e(smem + L::OFF_Q + x * L::Q_BYTES + h * HALF_BYTES, &p.map_q, q_full, h * 64, w.hq, w.q0 + x * BQ, w.b, leader);
+            tma_load_4d_e(smem + L::OFF_Q + x * L::Q_BYTES + h * HALF_BYTES, &p.map_q[w.layer], q_full, h * 64, w.hq, w.q0 + x * BQ, w.b, leader);
         auto load_k = [&](int j) -> bool {
           const int s = kg % FWD_KSTAGES;
           if (!mbar_wait(&k_empty[s], ((kg / FWD_KSTAGES) & 1) ^ 1, err)) return false;
           mbar_expect_tx_e(&k_full[s], L::KV_BYTES, leader);
 #pragma unroll
           for (int h = 0; h < HALVES; ++h)
-            tma_load_4d_e(smem + L::OFF_K + s * L::KV_BYTES + h * HALF_BYTES, &p.map_k, &k_full[s], h * 64, w.hk, j * BKV, w.b, leader);
+            tma_load_4d_e(smem + L::OFF_K + s * L::KV_BYTES + h * HALF_BYTES, &p.map_k[w.layer], &k_full[s], h * 64, w.hk, j * BKV, w.b, leader);
           ++kg;
           return true;
         };
@@ -199,7 +201,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
           mbar_expect_tx_e(&v_full[s], L::KV_BYTES, leader);
 #pragma unroll
           for (int h = 0; h < HALVES; ++h)
-            tma_load_4d_e(smem + L::OFF_V + s * L::KV_BYTES + h * HALF_BYTES, &p.map_v, &v_full[s], h * 64, w.hk, j * BKV, w.b, leader);
+            tma_load_4d_e(smem + L::OFF_V + s * L::KV_BYTES + h * HALF_BYTES, &p.map_v[w.layer], &v_full[s], h * 64, w.hk, j * BKV, w.b, leader);
           ++vg;
           return true;
         };
@@ -403,7 +405,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
         const float l_sum = (f2_lo(l2) + f2_hi(l2)) + (f2_lo(l2b) + f2_hi(l2b));
         const float inv_l = 1.f / l_sum;
         const bool valid = q_row < p.S;
-        __nv_bfloat16* dst = p.o + ((size_t(w.b) * p.S + (valid ? q_row : 0)) * p.Hq + w.hq) * DH;
+        __nv_bfloat16* dst = p.o[w.layer] + ((size_t(w.b) * p.S + (valid ? q_row : 0)) * p.Hq + w.hq) * DH;
 #pragma unroll
         for (int g = 0; g < DH / 32; ++g) {
           uint32_t tmp[32];
@@ -425,7 +427,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) attn_fwd_kernel(const __grid_c
             }
           }
         }
-        if (valid) p.lse[(size_t(w.b) * p.Hq + w.hq) * p.S + q_row] = (m_used + log2f(l_sum)) * 0.6931471805599453f;
+        if (valid) p.lse[w.layer][(size_t(w.b) * p.Hq + w.hq) * p.S + q_row] = (m_used + log2f(l_sum)) * 0.6931471805599453f;
       } else if (ok) {
         mbar_arrive(&o_free[x]);  // this query tile does not exist in this item: nothing to read out
       }
@@ -461,16 +463,21 @@ int attn_fwd_read_status() {
   return v;
 }
 
-// One layer: q [B,S,Hq,dh], k/v [B,S,Hkv,dh] of the layer's donor.
-int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, const void* k, const void* v, void* o,
-                   float* lse, cudaStream_t stream) {
-  FwdParams p;
-  int rc = make_map_bshd(&p.map_q, q, s->B, s->S, s->Hq, s->dh, BQ);
-  if (rc == KVP_OK) rc = make_map_bshd(&p.map_k, k, s->B, s->S, s->Hkv, s->dh, BKV);
-  if (rc == KVP_OK) rc = make_map_bshd(&p.map_v, v, s->B, s->S, s->Hkv, s->dh, BKV);
-  if (rc != KVP_OK) return rc;
-  p.o = reinterpret_cast<__nv_bfloat16*>(o);
-  p.lse = lse;
+// n layers (at most FWD_MAX_LAYERS) in one launch: q[i] [B,S,Hq,dh], k[i] / v[i] [B,S,Hkv,dh] of layer i's donor.
+int attn_fwd_layers(const kvp_shape* s, int causal, float scale, const void* const* q, const void* const* k,
+                    const void* const* v, void* const* o, float* const* lse, int n, cudaStream_t stream) {
+  if (n < 1 || n > FWD_MAX_LAYERS) return KVP_ERR_INVALID_ARG;
+  static thread_local FwdParams p;   // 3 KB of tensor maps: kept off the stack
+  for (int i = 0; i < FWD_MAX_LAYERS; ++i) {
+    const int l = i < n ? i : 0;
+    int rc = make_map_bshd(&p.map_q[i], q[l], s->B, s->S, s->Hq, s->dh, BQ);
+    if (rc == KVP_OK) rc = make_map_bshd(&p.map_k[i], k[l], s->B, s->S, s->Hkv, s->dh, BKV);
+    if (rc == KVP_OK) rc = make_map_bshd(&p.map_v[i], v[l], s->B, s->S, s->Hkv, s->dh, BKV);
+    if (rc != KVP_OK) return rc;
+    p.o[i] = reinterpret_cast<__nv_bfloat16*>(o[l]);
+    p.lse[i] = lse[l];
+  }
+  p.n_layers = n;
   p.B = s->B;
   p.S = s->S;
   p.Hq = s->Hq;
@@ -479,17 +486,19 @@ int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, c
   const float sc = scale == 0.f ? 1.f / sqrtf(float(s->dh)) : scale;
   p.scale_log2 = sc * 1.4426950408889634f;
   const int n_qtiles = (s->S + BQ - 1) / BQ;
-  const int n_items = s->B * s->Hq * ((n_qtiles + 1) / 2);
-  const int grid = min(n_items, sm_count());   // persistent: one CTA per SM walks a list of (b, hq, tile pair) items
-  cudaError_t e;
+  const long long n_items = (long long)n * s->B * s->Hq * ((n_qtiles + 1) / 2);
+  if (n_items > 0x7fffffffLL) return KVP_ERR_UNSUPPORTED;
+  // persistent: one CTA per SM walks a list of (layer, b, hq, tile pair) items
+  const int grid = int(n_items < (long long)sm_count() ? n_items : (long long)sm_count());
+  static const cudaError_t attr128 =
+      cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::TOTAL);
+  static const cudaError_t attr64 =
+      cudaFuncSetAttribute(attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::TOTAL);
+  if (attr128 != cudaSuccess || attr64 != cudaSuccess) return KVP_ERR_CUDA;
   timing_before(KVP_KERNEL_ATTN_FWD, stream);
   if (s->dh == 128) {
-    e = cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::TOTAL);
-    if (e != cudaSuccess) return KVP_ERR_CUDA;
     attn_fwd_kernel<128><<<grid, FWD_THREADS, FwdSmem<128>::TOTAL, stream>>>(p);
   } else if (s->dh == 64) {
-    e = cudaFuncSetAttribute(attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::TOTAL);
-    if (e != cudaSuccess) return KVP_ERR_CUDA;
     attn_fwd_kernel<64><<<grid, FWD_THREADS, FwdSmem<64>::TOTAL, stream>>>(p);
   } else {
     return KVP_ERR_UNSUPPORTED;
@@ -498,5 +507,7 @@ int attn_fwd_layer(const kvp_shape* s, int causal, float scale, const void* q, c
   note_launch();
   return cudaGetLastError() == cudaSuccess ? KVP_OK : KVP_ERR_CUDA;
 }
+
+int attn_fwd_max_layers() { return FWD_MAX_LAYERS; }
 
 }  // namespace kvp

@@ -245,6 +245,9 @@ SHAPES = [
     (1, 65, 2, 1, 128, [0, 0], False),
     (3, 200, 6, 3, 128, [0, 0, 0, 0, 0, 0, 0, 0], True),    # the largest donor group (8 layers), odd pair count
     (2, 193, 4, 4, 64, [0, 1, 1, 3], False),                # MHA (G = 1), mixed groups
+    (1, 130, 2, 1, 64, [0, 0, 0, 3, 3, 5, 5, 5, 8, 8], True),  # ten layers: two forward launches (eight + two)
+    (3, 2100, 6, 3, 64, [0, 0], True),                      # 324 forward work items on 148 persistent CTAs: three
+                                                            # rounds, the last one short and dealt out backwards
 ]
 
 

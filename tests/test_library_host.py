@@ -63,6 +63,22 @@ def test_workspace_queries_and_argument_validation_without_gpu(kvp):
     assert kvp.decode_workspace_bytes(kvp.DecodeDesc(4, 2, 8, 2, 128, 100, 10, 20), [0, 0, 2, 2]) == 0
 
 
+def test_self_tests_and_tile_mode_switch_validate_before_touching_the_device(kvp):
+    # both bounded-wait self-tests refuse a missing or too small scratch buffer before any launch
+    for fn, need in ((kvp.lib.kvp_selftest_bounded_wait, 512 * 1024), (kvp.lib.kvp_selftest_bounded_wait_pair, 768 * 1024)):
+        assert fn(None, need, None) == kvp.ERR_WORKSPACE
+        assert fn(0x1000, need - 1, None) == kvp.ERR_WORKSPACE
+        assert fn(0x1008, need, None) == kvp.ERR_WORKSPACE          # not 16-byte aligned
+    # the pair self-test is refused while CTA pairs are switched off; the switch clamps its argument
+    try:
+        kvp.set_gemm_pair_mode(0)
+        assert kvp.lib.kvp_selftest_bounded_wait_pair(0x1000, 768 * 1024, None) == kvp.ERR_UNSUPPORTED
+        kvp.set_gemm_pair_mode(7)
+        kvp.set_gemm_pair_mode(-3)
+    finally:
+        kvp.set_gemm_pair_mode(1)
+
+
 def _rand_instance(rng):
     Pn = rng.randint(1, 6)
     sizes = [rng.randint(1, 5) for _ in range(Pn)]

@@ -539,6 +539,8 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
         "config": {"workload": cfg.name, "layers": cfg.L, "donor": cfg.donor, "batch_per_gpu": cfg.B,
                    "global_batch": cfg.B * world, "seq_len": cfg.S, "d_model": cfg.D, "heads": [cfg.Hq, cfg.Hkv],
                    "head_dim": cfg.dh, "parallelism": f"dp{world}", "l2": "inputs larger than L2 (about 10 GB live)",
+                   "gemm_tiles": {0: "single-CTA 128x256 everywhere", 1: "CTA pairs 256x256 for the forward GEMMs, single-CTA "
+                                  "128x256 for the gradient GEMMs", 2: "CTA pairs 256x256 everywhere"}[args.gemm_pair_mode],
                    "flops": "value: attention kernels only, model count (forward 2 GEMMs, backward 4), causal pairs "
                             "S(S+1)/2, over the summed device time of the attention kernels inside the timed block step; "
                             "ms_per_step: the whole block step (projections + attention)"},

@@ -303,6 +303,18 @@ class TrainRunner:
         torch.cuda.empty_cache()
 
 
+def train_config(cfg: W.TrainCfg, world: int, gemm_pair_mode: int) -> dict:
+    """The `config` object of a training / prefill line; the reference arm prints the same one."""
+    return {"workload": cfg.name, "layers": cfg.L, "donor": cfg.donor, "batch_per_gpu": cfg.B,
+            "global_batch": cfg.B * world, "seq_len": cfg.S, "d_model": cfg.D, "heads": [cfg.Hq, cfg.Hkv],
+            "head_dim": cfg.dh, "parallelism": f"dp{world}", "l2": "inputs larger than L2 (about 10 GB live)",
+            "gemm_tiles": {0: "single-CTA 128x256 everywhere", 1: "CTA pairs 256x256 for the forward GEMMs, single-CTA "
+                           "128x256 for the gradient GEMMs", 2: "CTA pairs 256x256 everywhere"}[gemm_pair_mode],
+            "flops": "value: attention kernels only, model count (forward 2 GEMMs, backward 4), causal pairs "
+                     "S(S+1)/2, over the summed device time of the attention kernels inside the timed block step; "
+                     "ms_per_step: the whole block step (projections + attention)"}
+
+
 def cpu_baseline_train(cfg: W.TrainCfg, backward: bool, heads: int = 4, proj_tokens: int = 1024):
     """The oracle, as it stands, on a bounded exact slice: attention forward (+ backward) of one
     layer, one sequence, `heads` query heads of one KV group at the full sequence length, and the
@@ -536,14 +548,7 @@ def run_train_like(args, kvp, rank, local_rank, world, device, peaks, peaks_kind
         "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "layers": cfg.L, "donor": cfg.donor, "batch_per_gpu": cfg.B,
-                   "global_batch": cfg.B * world, "seq_len": cfg.S, "d_model": cfg.D, "heads": [cfg.Hq, cfg.Hkv],
-                   "head_dim": cfg.dh, "parallelism": f"dp{world}", "l2": "inputs larger than L2 (about 10 GB live)",
-                   "gemm_tiles": {0: "single-CTA 128x256 everywhere", 1: "CTA pairs 256x256 for the forward GEMMs, single-CTA "
-                                  "128x256 for the gradient GEMMs", 2: "CTA pairs 256x256 everywhere"}[args.gemm_pair_mode],
-                   "flops": "value: attention kernels only, model count (forward 2 GEMMs, backward 4), causal pairs "
-                            "S(S+1)/2, over the summed device time of the attention kernels inside the timed block step; "
-                            "ms_per_step: the whole block step (projections + attention)"},
+        "config": train_config(cfg, world, args.gemm_pair_mode),
         "clocks": clocks, "gpu_launches": int(launches),
         "attn_ms_per_step": attn_ms,
         "attn_flash_convention_tflops": flash,
@@ -947,13 +952,15 @@ def reference_arm(args, rank, world):
     steps, warmup = args.steps, args.warmup
     if args.workload == "decode":
         fn = lambda: cpu_baseline_decode(W.C3, n_seq=1)
-        metric, cfgname = "shared-cache decode tokens/s", W.C3.name
+        metric = "shared-cache decode tokens/s"
+        config = {"workload": W.C3.name, "note": "fp64 CPU oracle on a bounded sample per step"}
     else:
+        # the same workload, config object and sample as the cpu_baseline of the CUDA arm's line
         backward = args.workload != "prefill"
         cfg = W.C2 if backward else W.C1
-        fn = lambda: cpu_baseline_train(cfg, backward, heads=1, proj_tokens=256)
+        fn = lambda: cpu_baseline_train(cfg, backward)
         metric = "shared-KV attn fwd+bwd TFLOP/s" if backward else "shared-KV attn prefill fwd TFLOP/s"
-        cfgname = cfg.name
+        config = train_config(cfg, world, args.gemm_pair_mode)
     for _ in range(min(warmup, 1)):
         fn()
     t0 = time.perf_counter()
@@ -967,7 +974,7 @@ def reference_arm(args, rank, world):
     line = {"impl": "reference", "metric": metric, "value": value, "unit": last["unit"], "n_gpus": world,
             "steps": steps, "warmup": min(warmup, 1), "ms_per_step": dt / steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfgname, "note": "fp64 CPU oracle on a bounded sample per step"},
+            "config": config,
             "cpu_baseline": {"value": value, "unit": last["unit"], "cores": last["cores"], "kind": "oracle",
                              "sample": last["sample"]},
             "e2e": {"value": value, "unit": last["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}

@@ -72,16 +72,17 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(const uint4* __re
 }
 
 // In-place rotary embedding of x [B, S, H, dh]: pair i of every head turns by (pos0 + s) * theta^(-2i/dh).
-// One thread per 8 consecutive elements (4 pairs).  The frequencies arrive as float pairs hi + lo rounded from
-// the host's double values; the angle pos * f is formed as an exact product p = pos * hi plus its rounding
-// error and the lo term, sine and cosine of the float p are taken after an exact range reduction, and the small remainder is
-// applied as a second-order rotation (|remainder| <= half an ulp of p, below 2^-6 for the positions < 2^18
-// the entry point admits, so the neglected third-order term is under 1e-6).
-constexpr int kMaxRopePairs = 128;  // dh <= 256
+// One thread per (token, 8 consecutive elements of the head dimension): it forms the four rotations once and
+// applies them to that slice of EVERY head of the token, so the sines and cosines cost 1/H of a per-element
+// evaluation and the kernel is left with its loads and stores.  The frequencies arrive as float pairs hi + lo
+// rounded from the host's double values; the angle pos * f is formed as an exact product p = pos * hi plus its
+// rounding error and the lo term, sine and cosine of the float p are taken after an exact range reduction, and the
+// small remainder is applied as a second-order correction.
+constexpr int kMaxRopePairs = 128;
 struct RopeFreq {
   float2 f[kMaxRopePairs];
 };
-__global__ void rope_kernel(uint4* __restrict__ x, uint32_t n8, uint32_t S, uint32_t per_tok, uint32_t dh8, int pos0,
+__global__ void rope_kernel(uint4* __restrict__ x, uint32_t n_work, uint32_t S, uint32_t H, uint32_t dh8, int pos0,
                             const __grid_constant__ RopeFreq fr) {
   // lanes of a warp need different table entries: shared memory serves them in one pass, the constant bank
   // that holds kernel parameters would replay once per distinct address
@@ -89,13 +90,12 @@ __global__ void rope_kernel(uint4* __restrict__ x, uint32_t n8, uint32_t S, uint
   for (int k = threadIdx.x; k < kMaxRopePairs; k += blockDim.x) freq[k] = fr.f[k];
   __syncthreads();
   const uint32_t stride = gridDim.x * blockDim.x;
-  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {  // 32-bit index arithmetic only
+  const uint32_t per_tok = H * dh8;
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n_work; i += stride) {  // 32-bit index arithmetic only
     const uint32_t c = i % dh8;                       // which group of 4 pairs inside the head
-    const uint32_t tok = i / per_tok;                 // b * S + s
+    const uint32_t tok = i / dh8;                     // b * S + s
     const float pos = float(pos0 + int(tok % S));     // exact
-    float f[8];
-    uint4 v = x[i];
-    unpack8(v, f);
+    float sn2[4], cs2[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float2 fq = freq[c * 4 + k];
@@ -109,12 +109,31 @@ __global__ void rope_kernel(uint4* __restrict__ x, uint32_t n8, uint32_t S, uint
       rr = fmaf(-kk, 5.070363386039389e-06f, rr);
       const float sn = __sinf(rr), cs = __cosf(rr);
       const float h = 0.5f * d * d;
-      const float sn2 = sn + d * cs - h * sn, cs2 = cs - d * sn - h * cs;
-      const float a = f[2 * k], b = f[2 * k + 1];
-      f[2 * k] = a * cs2 - b * sn2;
-      f[2 * k + 1] = a * sn2 + b * cs2;
+      sn2[k] = sn + d * cs - h * sn;
+      cs2[k] = cs - d * sn - h * cs;
     }
-    x[i] = pack8(f);
+    uint4* const base = x + size_t(tok) * per_tok + c;
+    constexpr uint32_t UNROLL = 4;   // loads in flight per thread
+    for (uint32_t h0 = 0; h0 < H; h0 += UNROLL) {
+      uint4 v[UNROLL];
+#pragma unroll
+      for (uint32_t u = 0; u < UNROLL; ++u)
+        if (h0 + u < H) v[u] = base[size_t(h0 + u) * dh8];
+#pragma unroll
+      for (uint32_t u = 0; u < UNROLL; ++u) {
+        if (h0 + u < H) {
+          float f[8];
+          unpack8(v[u], f);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float a = f[2 * k], b = f[2 * k + 1];
+            f[2 * k] = a * cs2[k] - b * sn2[k];
+            f[2 * k + 1] = a * sn2[k] + b * cs2[k];
+          }
+          base[size_t(h0 + u) * dh8] = pack8(f);
+        }
+      }
+    }
   }
 }
 
@@ -178,9 +197,9 @@ extern "C" int kvp_rope(int32_t B, int32_t S, int32_t H, int32_t dh, float theta
   if (per_seq >= (size_t(1) << 31)) return KVP_ERR_UNSUPPORTED;
   const int seqs_per_launch = int(std::max<size_t>(1, ((size_t(1) << 31) - 1) / per_seq));
   for (int b0 = 0; b0 < B; b0 += seqs_per_launch) {
-    const uint32_t m8 = uint32_t(size_t(std::min(seqs_per_launch, B - b0)) * per_seq);
-    rope_kernel<<<streaming_blocks(m8, 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-        reinterpret_cast<uint4*>(x) + size_t(b0) * per_seq, m8, uint32_t(S), uint32_t(H) * (dh / 8), uint32_t(dh / 8), pos0, fr);
+    const uint32_t n_work = uint32_t(size_t(std::min(seqs_per_launch, B - b0)) * S * (dh / 8));   // (token, 8-element slice)
+    rope_kernel<<<streaming_blocks(n_work, 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<uint4*>(x) + size_t(b0) * per_seq, n_work, uint32_t(S), uint32_t(H), uint32_t(dh / 8), pos0, fr);
     note_launch();
   }
   return cudaGetLastError() == cudaSuccess ? KVP_OK : KVP_ERR_CUDA;

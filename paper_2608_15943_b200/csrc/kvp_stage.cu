@@ -32,15 +32,26 @@ constexpr int kMaxChunks = 4;  // D <= 8192
 __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w,
                                                                uint4* __restrict__ y, int T, int D8, float inv_d, float eps) {
   __shared__ float part[kNormThreads / 32];
-  for (int row = blockIdx.x; row < T; row += gridDim.x) {
+  auto load_row = [&](int row, uint4 (&v)[kMaxChunks]) {
     const uint4* xr = x + size_t(row) * D8;
-    uint4 v[kMaxChunks];
+#pragma unroll
+    for (int c = 0; c < kMaxChunks; ++c) {
+      const int i = c * kNormThreads + threadIdx.x;
+      if (i < D8) v[c] = xr[i];
+    }
+  };
+  uint4 v[kMaxChunks], vn[kMaxChunks];
+  if (int(blockIdx.x) < T) load_row(blockIdx.x, v);
+  for (int row = blockIdx.x; row < T; row += gridDim.x) {
+    // the next row of this CTA is requested before the current one is reduced: its latency hides under the two
+    // block barriers and the stores of this row
+    const int next = row + gridDim.x;
+    if (next < T) load_row(next, vn);
     float ss = 0.f;
 #pragma unroll
     for (int c = 0; c < kMaxChunks; ++c) {
       const int i = c * kNormThreads + threadIdx.x;
       if (i < D8) {
-        v[c] = xr[i];
         float f[8];
         unpack8(v[c], f);
 #pragma unroll
@@ -68,6 +79,8 @@ __global__ void __launch_bounds__(kNormThreads) rmsnorm_kernel(const uint4* __re
         y[size_t(row) * D8 + i] = pack8(f);
       }
     }
+#pragma unroll
+    for (int c = 0; c < kMaxChunks; ++c) v[c] = vn[c];
   }
 }
 
